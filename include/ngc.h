@@ -1,0 +1,204 @@
+/*
+ * ngc.h -- C ABI of the nested-gradient-code (NGC) hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library simulates, on one GPU, one iteration of coded distributed gradient
+ * descent with the nested gradient code of arXiv 2212.08580 ("Nested Gradient Codes
+ * for Straggler Mitigation in Distributed Machine Learning"):
+ *
+ *   workers:    partial gradients g_j of the k data partitions (Section II-C),
+ *               coded responses   x_i = b^(i) G,  X = B G      (Section II-C),
+ *   main node:  choice of the component code and of the responsive set S by the
+ *               progress-tracking / termination-message rule   (Sections II-D, III),
+ *               decoding vector a with supp(a) in S, a B = 1   (Definition 1),
+ *               decoded gradient  g = sum_{i in S} a_i x_i     (Section II-C).
+ *
+ * Conventions
+ *   - Every function returns an int status: 0 = NGC_OK, negative = error (below).
+ *     No exceptions, no abort, no device-side traps.
+ *   - "host" pointers are ordinary CPU memory; "dev" pointers are CUDA device memory
+ *     on the current device.  The caller owns every buffer it passes in.  The plan
+ *     owns its tables and a device workspace that it allocates on first use and frees
+ *     in ngc_plan_destroy.
+ *   - `cuda_stream` is a cudaStream_t cast to void* (NULL = legacy default stream).
+ *     Calls that take a stream only enqueue work and return; results are valid after
+ *     the stream has been synchronised.  Calls on one plan must not overlap on the GPU
+ *     (they share the plan's workspace).
+ *   - Indices are 0-based and cyclic mod n: worker i at tolerance s holds partitions
+ *     i, i+1, ..., i+s (mod n).
+ */
+#ifndef NGC_H
+#define NGC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NGC_MAX_N 128 /* workers */
+#define NGC_MAX_S 32  /* largest straggler tolerance */
+#define NGC_MAX_LEVELS 16
+
+enum {
+  NGC_OK = 0,
+  NGC_ERR_INVALID = -1,     /* bad argument: sizes, ordering, null pointer, misaligned pointer, unsupported shape */
+  NGC_ERR_UNDECODABLE = -2, /* more than s_L workers never finish: no component code becomes decodable */
+  NGC_ERR_SINGULAR = -3,    /* decoding vector residual |a B - 1| above threshold */
+  NGC_ERR_CUDA = -4,        /* a CUDA runtime call failed; see ngc_last_cuda_error */
+  NGC_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reported by ngc_device_status) */
+  NGC_ERR_NOMEM = -6        /* host allocation failed */
+};
+
+typedef enum { NGC_LSQ = 0, NGC_LOGISTIC = 1, NGC_SOFTMAX = 2, NGC_MLP = 3 } ngc_model_kind;
+typedef enum { NGC_F32 = 0, NGC_BF16 = 1, NGC_F64 = 2 } ngc_dtype;
+
+/*
+ * The function f(d, theta) whose loss gradient is distributed (Section II-B).  The
+ * paper leaves the loss open; the four kinds are least squares 1/2 (x.theta - y)^2,
+ * logistic regression (labels 0/1), softmax regression (theta = W in R^{d x C},
+ * row-major) and a one-hidden-layer ReLU network with softmax cross-entropy (theta =
+ * [W1 (d x hidden, row-major), b1, W2 (hidden x C), b2]).  Gradients are SUMS over a
+ * partition's rows (the 1/m sits in the update rule, Eq. 1).
+ */
+typedef struct {
+  int32_t kind;               /* ngc_model_kind */
+  int32_t x_dtype;            /* NGC_F32 or NGC_BF16: storage type of the data matrix */
+  int32_t rows_per_partition; /* m / k */
+  int32_t d;                  /* features (columns of the data matrix) */
+  int32_t n_classes;          /* C, softmax / MLP only */
+  int32_t hidden;             /* MLP only */
+} ngc_model_t;
+
+typedef struct ngc_plan_s ngc_plan_t; /* opaque */
+
+/* Result of the stopping rule for one straggler pattern. */
+typedef struct {
+  int32_t layer;                 /* index l of the chosen component code */
+  int32_t sigma;                 /* its tolerance s_l */
+  int32_t nS;                    /* n - s_l */
+  int32_t S[NGC_MAX_N];          /* responsive set, increasing worker index */
+  double latency;                /* gamma + eps + instant the component became decodable */
+  int32_t tasks_done[NGC_MAX_N]; /* partial gradients each worker had finished by then */
+} ngc_step_info_t;
+
+/* Parameter count l of a model (length of theta and of every gradient); <0 on a bad descriptor. */
+int64_t ngc_num_params(const ngc_model_t *model);
+
+/*
+ * Algorithm 1 (construction of an (n, k, s_max) nested gradient code), for the listed
+ * tolerances s_levels[0] < ... < s_levels[n_levels-1], each in [0, n).  Tolerance 0
+ * gives B = I.  n_partitions must be a multiple of n_workers; k = q n is handled as n
+ * atomic tasks of q consecutive partitions (Section II-C).  Coefficients follow the
+ * cyclic-repetition scheme the paper cites: row i of B_s is supported on the window
+ * i..i+s, has b_ii = 1 and lies in the null space of an s x n matrix H with zero row
+ * sums whose entries are drawn from the SplitMix64 stream of `seed`.  gamma / eps are
+ * the constant communication and signalling delays of Section II-D, only added to the
+ * reported latency.  Pure host computation in a fixed operation order (results are
+ * bit-reproducible); no GPU is touched.  *out is owned by the library.
+ */
+int ngc_plan(int n_workers, int n_levels, const int *s_levels, int n_partitions, uint64_t seed,
+             double gamma, double eps, ngc_plan_t **out);
+void ngc_plan_destroy(ngc_plan_t *plan);
+
+/*
+ * Introspection (host pointers, valid until ngc_plan_destroy).
+ * ngc_plan_B: *coef points to n x (s+1) doubles, row i = B_s[i, i], B_s[i, i+1], ..., B_s[i, i+s]
+ * (columns mod n); *width = s + 1.
+ * ngc_plan_schedule: *order is n x (s_L+1) partition-group ids in execution order
+ * (Section III, layered task scheduling); *tasks_per_layer has n_levels entries s_l + 1.
+ */
+int ngc_plan_B(const ngc_plan_t *plan, int layer, const double **coef, int *width);
+int ngc_plan_schedule(const ngc_plan_t *plan, const int32_t **order, const int32_t **tasks_per_layer);
+
+/*
+ * Storage type of the coded gradients x_i: NGC_F64, NGC_F32, or -1 = automatic (F64
+ * for least squares / logistic, F32 for softmax / MLP).  The code matrices are
+ * ill-conditioned for large n and s, so F32 storage costs accuracy.
+ */
+int ngc_set_coded_dtype(ngc_plan_t *plan, int dtype);
+int ngc_coded_dtype(const ngc_plan_t *plan, const ngc_model_t *model);
+
+/*
+ * Stopping and signalling rule (Section II-D last paragraph; Section III last
+ * paragraph; proof of Theorem 1): task_times_host is n x (s_L+1) doubles, entry
+ * [i][m] the duration of worker i's (m+1)-th task, +inf = never finishes.  Component
+ * s_l becomes decodable when n - s_l workers have finished s_l + 1 tasks; the earliest
+ * such instant wins (ties: smaller l), and exactly n - s_l responders are kept
+ * (earliest first, ties by worker index).  Host only.  NGC_ERR_UNDECODABLE if no
+ * component ever becomes decodable.
+ */
+int ngc_select(const ngc_plan_t *plan, const double *task_times_host, ngc_step_info_t *info);
+
+/*
+ * Workers' side of one iteration (Section II-C): partial gradients of all partitions
+ * at theta, and the coded responses of all n workers for component `layer`.
+ *   theta_dev : l floats.
+ *   X_dev     : [k][rows_per_partition][d], row-major, contiguous, model->x_dtype; 16-byte aligned.
+ *   y_dev     : [k][rows_per_partition]; float targets / 0-1 labels (LSQ, LOGISTIC) or int32 class ids.
+ *   coded_dev : out, [n][l] in ngc_coded_dtype(plan, model); row i is x_i.
+ * Each partition is read from device memory once; every g_j is computed once and fanned
+ * out to the s_l + 1 workers that hold it.
+ */
+int ngc_grad_encode(ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev, const void *X_dev,
+                    const void *y_dev, int layer, void *coded_dev, void *cuda_stream);
+
+/*
+ * Decoding vectors (Definition 1: a row of A with support in S and a B = 1), computed
+ * on the device by a batched fp64 solve.  S lists responsive workers in increasing
+ * order, nS >= n - s_l; if nS is larger, the n - s_l smallest indices are used, which
+ * makes a unique.  a_host_out receives n doubles (zero off the used set).  Synchronous.
+ * ngc_decode_vectors: `batch` patterns, S_host is batch x nS, a_host_out batch x n.
+ */
+int ngc_decode_vector(ngc_plan_t *plan, int layer, const int32_t *S_host, int nS, double *a_host_out);
+int ngc_decode_vectors(ngc_plan_t *plan, int layer, const int32_t *S_host, int nS, int batch,
+                       double *a_host_out, double *residual_host_out /* batch, may be NULL */);
+
+/*
+ * Main node's decode (Section II-C): g = sum_{i in S} a_i x_i with a from the solve
+ * above.  coded_dev is [n][l] as written by ngc_grad_encode for the same layer;
+ * grad_dev receives l floats.  Asynchronous on the stream.
+ */
+int ngc_decode(ngc_plan_t *plan, int layer, const int32_t *S_host, int nS, const void *coded_dev,
+               int coded_dtype, int64_t l, float *grad_dev, void *cuda_stream);
+
+/*
+ * One full iteration for a given straggler pattern: ngc_select on the host, then
+ * ngc_grad_encode for the chosen component and ngc_decode over its responsive set,
+ * enqueued on the stream.  coded_dev is caller-provided scratch of n x l coded values.
+ */
+int ngc_step(ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev, const void *X_dev,
+             const void *y_dev, const double *task_times_host, void *coded_dev, float *grad_dev,
+             ngc_step_info_t *info, void *cuda_stream);
+
+/*
+ * Same iteration with every buffer in HOST memory: copies theta, X, y to the device,
+ * runs ngc_step, copies the decoded gradient back and synchronises.  Device staging
+ * buffers belong to the plan and are reused across calls.
+ */
+int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta_host, const void *X_host,
+                  const void *y_host, const double *task_times_host, float *grad_host, ngc_step_info_t *info);
+
+/*
+ * Response-time model of Section II-D (Eq. 2 without the constants): task_times_host
+ * [n][tasks] = shift + Exp(rate) i.i.d. from the SplitMix64 stream of `seed`; each
+ * worker fails (all entries +inf) independently with probability p_fail.  Host only.
+ */
+int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate, double p_fail,
+                     double *task_times_host);
+
+/* Bytes of device workspace the plan currently holds. */
+size_t ngc_workspace_bytes(const ngc_plan_t *plan);
+/* Synchronises the device and returns NGC_OK or NGC_ERR_TIMEOUT / NGC_ERR_SINGULAR from the status
+ * words the kernels of this plan wrote; *residual_out (may be NULL) gets the largest decode residual seen. */
+int ngc_device_status(ngc_plan_t *plan, double *residual_out);
+/* cudaError_t of the last failed runtime call on this plan (0 if none). */
+int ngc_last_cuda_error(const ngc_plan_t *plan);
+/* How many kernels of this library the plan has launched so far. */
+int64_t ngc_launch_count(const ngc_plan_t *plan);
+const char *ngc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NGC_H */

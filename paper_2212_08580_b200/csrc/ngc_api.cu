@@ -1,0 +1,290 @@
+// C-ABI entry points that touch the GPU: argument checks, lazily created device tables and
+// workspace, and the launch sequences of the hot path.
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "ngc_device.h"
+
+namespace ngc {
+int device_sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+}  // namespace ngc
+
+namespace {
+
+#define NGC_CUDA(p, call)                      \
+  do {                                         \
+    cudaError_t e__ = (call);                  \
+    if (e__ != cudaSuccess) {                  \
+      (p)->last_cuda = (int)e__;               \
+      return NGC_ERR_CUDA;                     \
+    }                                          \
+  } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int ensure_tables(ngc_plan_s *p) {
+  if (p->tables_on_device) return NGC_OK;
+  int dev = 0;
+  NGC_CUDA(p, cudaGetDevice(&dev));
+  p->device = dev;
+  for (auto &lv : p->lv) {
+    NGC_CUDA(p, cudaMalloc(&lv.d_coef, lv.coef.size() * sizeof(double)));
+    NGC_CUDA(p, cudaMemcpy(lv.d_coef, lv.coef.data(), lv.coef.size() * sizeof(double), cudaMemcpyHostToDevice));
+    NGC_CUDA(p, cudaMalloc(&lv.d_a0, lv.a0.size() * sizeof(double)));
+    NGC_CUDA(p, cudaMemcpy(lv.d_a0, lv.a0.data(), lv.a0.size() * sizeof(double), cudaMemcpyHostToDevice));
+    if (!lv.N.empty()) {
+      NGC_CUDA(p, cudaMalloc(&lv.d_N, lv.N.size() * sizeof(double)));
+      NGC_CUDA(p, cudaMemcpy(lv.d_N, lv.N.data(), lv.N.size() * sizeof(double), cudaMemcpyHostToDevice));
+    }
+  }
+  NGC_CUDA(p, cudaMalloc(&p->d_status, 2 * sizeof(int)));
+  NGC_CUDA(p, cudaMemset(p->d_status, 0, 2 * sizeof(int)));
+  NGC_CUDA(p, cudaMalloc(&p->d_maxres, sizeof(double)));
+  NGC_CUDA(p, cudaMemset(p->d_maxres, 0, sizeof(double)));
+  p->tables_on_device = true;
+  return NGC_OK;
+}
+
+int ensure_ws(ngc_plan_s *p, size_t bytes) {
+  if (bytes <= p->ws_bytes) return NGC_OK;
+  if (p->ws) {
+    NGC_CUDA(p, cudaDeviceSynchronize());
+    NGC_CUDA(p, cudaFree(p->ws));
+    p->ws = nullptr;
+    p->ws_bytes = 0;
+  }
+  NGC_CUDA(p, cudaMalloc(&p->ws, bytes));
+  p->ws_bytes = bytes;
+  return NGC_OK;
+}
+
+int ensure_batch(ngc_plan_s *p, int batch) {
+  if (batch <= p->a_batch_cap) return NGC_OK;
+  if (p->d_a) {
+    NGC_CUDA(p, cudaDeviceSynchronize());
+    cudaFree(p->d_a);
+    cudaFree(p->d_resid);
+    cudaFree(p->d_masks);
+    p->d_a = nullptr; p->d_resid = nullptr; p->d_masks = nullptr; p->a_batch_cap = 0;
+  }
+  NGC_CUDA(p, cudaMalloc(&p->d_a, (size_t)batch * p->n * sizeof(double)));
+  NGC_CUDA(p, cudaMalloc(&p->d_resid, (size_t)batch * sizeof(double)));
+  NGC_CUDA(p, cudaMalloc(&p->d_masks, (size_t)batch * 2 * sizeof(uint64_t)));
+  p->a_batch_cap = batch;
+  return NGC_OK;
+}
+
+int ensure_staging(ngc_plan_s *p, void **buf, size_t *have, size_t want) {
+  if (want <= *have) return NGC_OK;
+  if (*buf) {
+    NGC_CUDA(p, cudaDeviceSynchronize());
+    NGC_CUDA(p, cudaFree(*buf));
+    *buf = nullptr;
+    *have = 0;
+  }
+  NGC_CUDA(p, cudaMalloc(buf, want));
+  *have = want;
+  return NGC_OK;
+}
+
+// Checks a responsive set and packs it into a bit mask.
+int pack_set(const ngc_plan_s *p, int layer, const int32_t *S, int nS, uint64_t *mask) {
+  const int n = p->n, s = p->lv[layer].s;
+  if (!S || nS < n - s || nS > n) return NGC_ERR_INVALID;
+  mask[0] = mask[1] = 0;
+  for (int t = 0; t < nS; ++t) {
+    if (S[t] < 0 || S[t] >= n) return NGC_ERR_INVALID;
+    if (t > 0 && S[t] <= S[t - 1]) return NGC_ERR_INVALID;
+    mask[S[t] >> 6] |= 1ull << (S[t] & 63);
+  }
+  return NGC_OK;
+}
+
+int check_model(const ngc_plan_s *p, const ngc_model_t *m) {
+  if (!m || m->rows_per_partition < 1 || m->d < 1) return NGC_ERR_INVALID;
+  if (ngc_num_params(m) < 0) return NGC_ERR_INVALID;
+  if (m->x_dtype != NGC_F32 && m->x_dtype != NGC_BF16) return NGC_ERR_INVALID;
+  (void)p;
+  return NGC_OK;
+}
+
+// The residual |a B - 1| above which a decode is reported as NGC_ERR_SINGULAR.
+constexpr double kResidualLimit = 1e-6;
+
+}  // namespace
+
+extern "C" {
+
+void ngc_plan_destroy(ngc_plan_t *p) {
+  if (!p) return;
+  if (p->tables_on_device || p->ws || p->st_X) {
+    cudaDeviceSynchronize();
+    for (auto &lv : p->lv) {
+      cudaFree(lv.d_coef);
+      cudaFree(lv.d_a0);
+      cudaFree(lv.d_N);
+    }
+    cudaFree(p->ws);
+    cudaFree(p->d_a);
+    cudaFree(p->d_resid);
+    cudaFree(p->d_masks);
+    cudaFree(p->d_status);
+    cudaFree(p->d_maxres);
+    cudaFree(p->st_X);
+    cudaFree(p->st_y);
+    cudaFree(p->st_theta);
+    cudaFree(p->st_coded);
+    cudaFree(p->st_grad);
+  }
+  delete p;
+}
+
+int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
+                    void *coded, void *cuda_stream) {
+  if (!p || !theta || !X || !y || !coded || layer < 0 || layer >= p->L) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  if (!aligned16(X) || !aligned16(coded) || !aligned16(theta)) return NGC_ERR_INVALID;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  rc = ensure_tables(p);
+  if (rc != NGC_OK) return rc;
+  const int cdt = ngc_coded_dtype(p, m);
+  const ngc_level_t &lv = p->lv[layer];
+
+  if (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) {
+    const int vec = (m->x_dtype == NGC_F32) ? 4 : 8;
+    if (m->d % vec != 0 || m->d / vec > 4 * 512) return NGC_ERR_INVALID;  // rows must be whole 16-byte vectors
+    const int sms = ngc::device_sm_count();
+    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
+    const ngc::RowSplit split = ngc::make_row_split(p->n, (long long)p->q * m->rows_per_partition, sms);
+    rc = ensure_ws(p, (size_t)p->n * split.P * m->d * sizeof(float));
+    if (rc != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_gemv_pair(*m, split, X, static_cast<const float *>(y), static_cast<const float *>(theta),
+                                      static_cast<float *>(p->ws), p->d_status, stream));
+    NGC_CUDA(p, ngc::launch_combine_encode(split, static_cast<const float *>(p->ws), lv.d_coef, p->n, lv.s, m->d,
+                                           coded, cdt, stream));
+    p->launches += 2;
+    return NGC_OK;
+  }
+  return NGC_ERR_INVALID;  // softmax / MLP paths are not built yet
+}
+
+int ngc_decode_vectors(ngc_plan_t *p, int layer, const int32_t *S, int nS, int batch, double *a_out,
+                       double *resid_out) {
+  if (!p || !S || !a_out || layer < 0 || layer >= p->L || batch < 1) return NGC_ERR_INVALID;
+  std::vector<uint64_t> masks((size_t)batch * 2);
+  for (int b = 0; b < batch; ++b) {
+    const int rc = pack_set(p, layer, S + (size_t)b * nS, nS, &masks[2 * (size_t)b]);
+    if (rc != NGC_OK) return rc;
+  }
+  int rc = ensure_tables(p);
+  if (rc != NGC_OK) return rc;
+  rc = ensure_batch(p, batch);
+  if (rc != NGC_OK) return rc;
+  NGC_CUDA(p, cudaMemcpy(p->d_masks, masks.data(), masks.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
+  ngc::MaskArg none{{0, 0}};
+  NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, p->d_masks, none, batch, p->d_a, p->d_resid, nullptr, 0));
+  p->launches += 1;
+  NGC_CUDA(p, cudaMemcpy(a_out, p->d_a, (size_t)batch * p->n * sizeof(double), cudaMemcpyDeviceToHost));
+  std::vector<double> res(batch);
+  NGC_CUDA(p, cudaMemcpy(res.data(), p->d_resid, (size_t)batch * sizeof(double), cudaMemcpyDeviceToHost));
+  int status = NGC_OK;
+  for (int b = 0; b < batch; ++b) {
+    if (resid_out) resid_out[b] = res[b];
+    if (!(res[b] <= kResidualLimit)) status = NGC_ERR_SINGULAR;
+  }
+  return status;
+}
+
+int ngc_decode_vector(ngc_plan_t *p, int layer, const int32_t *S, int nS, double *a_out) {
+  return ngc_decode_vectors(p, layer, S, nS, 1, a_out, nullptr);
+}
+
+int ngc_decode(ngc_plan_t *p, int layer, const int32_t *S, int nS, const void *coded, int coded_dtype, int64_t l,
+               float *grad, void *cuda_stream) {
+  if (!p || !coded || !grad || layer < 0 || layer >= p->L || l < 1) return NGC_ERR_INVALID;
+  if (coded_dtype != NGC_F32 && coded_dtype != NGC_F64) return NGC_ERR_INVALID;
+  if (!aligned16(coded)) return NGC_ERR_INVALID;
+  ngc::MaskArg mask;
+  int rc = pack_set(p, layer, S, nS, mask.w);
+  if (rc != NGC_OK) return rc;
+  rc = ensure_tables(p);
+  if (rc != NGC_OK) return rc;
+  rc = ensure_batch(p, 1);
+  if (rc != NGC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
+  NGC_CUDA(p, ngc::launch_decode(coded, coded_dtype, p->d_a, p->n, l, grad, stream));
+  p->launches += 2;
+  return NGC_OK;
+}
+
+int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y,
+             const double *task_times, void *coded, float *grad, ngc_step_info_t *info, void *cuda_stream) {
+  if (!p || !info) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  rc = ngc_select(p, task_times, info);
+  if (rc != NGC_OK) return rc;
+  rc = ngc_grad_encode(p, m, theta, X, y, info->layer, coded, cuda_stream);
+  if (rc != NGC_OK) return rc;
+  return ngc_decode(p, info->layer, info->S, info->nS, coded, ngc_coded_dtype(p, m), ngc_num_params(m), grad,
+                    cuda_stream);
+}
+
+int ngc_step_host(ngc_plan_t *p, const ngc_model_t *m, const float *theta, const void *X, const void *y,
+                  const double *task_times, float *grad, ngc_step_info_t *info) {
+  if (!p || !theta || !X || !y || !grad || !info) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  const int64_t l = ngc_num_params(m);
+  const size_t xb = (size_t)p->k * m->rows_per_partition * m->d * (m->x_dtype == NGC_F32 ? 4 : 2);
+  const size_t yb = (size_t)p->k * m->rows_per_partition * 4;
+  const size_t cb = (size_t)p->n * l * (ngc_coded_dtype(p, m) == NGC_F64 ? 8 : 4);
+  if ((rc = ensure_staging(p, &p->st_X, &p->st_X_bytes, xb)) != NGC_OK) return rc;
+  if ((rc = ensure_staging(p, &p->st_y, &p->st_y_bytes, yb)) != NGC_OK) return rc;
+  if ((rc = ensure_staging(p, &p->st_theta, &p->st_theta_bytes, (size_t)l * 4)) != NGC_OK) return rc;
+  if ((rc = ensure_staging(p, &p->st_coded, &p->st_coded_bytes, cb)) != NGC_OK) return rc;
+  if ((rc = ensure_staging(p, &p->st_grad, &p->st_grad_bytes, (size_t)l * 4)) != NGC_OK) return rc;
+  cudaStream_t stream = 0;
+  NGC_CUDA(p, cudaMemcpyAsync(p->st_theta, theta, (size_t)l * 4, cudaMemcpyHostToDevice, stream));
+  NGC_CUDA(p, cudaMemcpyAsync(p->st_y, y, yb, cudaMemcpyHostToDevice, stream));
+  NGC_CUDA(p, cudaMemcpyAsync(p->st_X, X, xb, cudaMemcpyHostToDevice, stream));
+  rc = ngc_step(p, m, p->st_theta, p->st_X, p->st_y, task_times, p->st_coded, static_cast<float *>(p->st_grad), info,
+                stream);
+  if (rc != NGC_OK) return rc;
+  NGC_CUDA(p, cudaMemcpyAsync(grad, p->st_grad, (size_t)l * 4, cudaMemcpyDeviceToHost, stream));
+  NGC_CUDA(p, cudaStreamSynchronize(stream));
+  return NGC_OK;
+}
+
+size_t ngc_workspace_bytes(const ngc_plan_t *p) {
+  if (!p) return 0;
+  return p->ws_bytes + p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes + p->st_grad_bytes;
+}
+
+int ngc_device_status(ngc_plan_t *p, double *residual_out) {
+  if (!p) return NGC_ERR_INVALID;
+  if (residual_out) *residual_out = 0.0;
+  if (!p->tables_on_device) return NGC_OK;
+  NGC_CUDA(p, cudaDeviceSynchronize());
+  int st[2] = {0, 0};
+  double mr = 0.0;
+  NGC_CUDA(p, cudaMemcpy(st, p->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+  NGC_CUDA(p, cudaMemcpy(&mr, p->d_maxres, sizeof(mr), cudaMemcpyDeviceToHost));
+  if (residual_out) *residual_out = mr;
+  if (st[0] != 0) return NGC_ERR_TIMEOUT;
+  if (!(mr <= kResidualLimit)) return NGC_ERR_SINGULAR;
+  return NGC_OK;
+}
+
+int ngc_last_cuda_error(const ngc_plan_t *p) { return p ? p->last_cuda : 0; }
+int64_t ngc_launch_count(const ngc_plan_t *p) { return p ? p->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,177 @@
+// Main-node side of the nested gradient code:
+//   * decoding vectors (Definition 1: supp(a) inside the responsive set S, a B = 1), one warp
+//     per straggler pattern, fp64;
+//   * the decode itself, g = sum_{i in S} a_i x_i (Section II-C), a bandwidth-bound weighted
+//     reduction over the coded gradients.
+#include "ngc_device.h"
+
+namespace ngc {
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Decoding vector for one pattern.  With a0 a particular solution of B^T a = 1 and N an
+// orthonormal basis of {v : B^T v = 0} (both from the plan), every solution is a0 + N z; asking
+// it to vanish on the s unused workers T gives the s x s system  N[T,:] z = -a0[T].  Solved by
+// Gaussian elimination with partial pivoting, one matrix row per lane.
+// ------------------------------------------------------------------------------------------
+constexpr int kSolveWarps = 4;
+
+__global__ void __launch_bounds__(kSolveWarps * 32)
+decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, int n, int s,
+                    const double *__restrict__ a0, const double *__restrict__ Nmat, const double *__restrict__ coef,
+                    double *__restrict__ a_out, double *__restrict__ resid_out, double *maxres) {
+  __shared__ double M[kSolveWarps][NGC_MAX_S][NGC_MAX_S + 1];
+  __shared__ double zs[kSolveWarps][NGC_MAX_S];
+  __shared__ double as[kSolveWarps][NGC_MAX_N];
+  __shared__ int tlist[kSolveWarps][NGC_MAX_S];
+  __shared__ unsigned char used[kSolveWarps][NGC_MAX_N];
+
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int b = blockIdx.x * kSolveWarps + w;
+  if (b >= batch) return;
+  uint64_t m0, m1;
+  if (masks) { m0 = masks[2 * b]; m1 = masks[2 * b + 1]; }
+  else { m0 = one.w[0]; m1 = one.w[1]; }
+
+  if (lane == 0) {
+    int kept = 0, nt = 0;
+    for (int i = 0; i < n; ++i) {
+      const bool in = ((i < 64 ? (m0 >> i) : (m1 >> (i - 64))) & 1ull) != 0;
+      if (in && kept < n - s) { used[w][i] = 1; ++kept; }
+      else { used[w][i] = 0; if (nt < s) tlist[w][nt] = i; ++nt; }
+    }
+  }
+  __syncwarp();
+
+  if (s > 0) {
+    if (lane < s) {
+      const int row = tlist[w][lane];
+      for (int c = 0; c < s; ++c) M[w][lane][c] = Nmat[(size_t)row * s + c];
+      M[w][lane][s] = -a0[row];
+    }
+    __syncwarp();
+    for (int p = 0; p < s; ++p) {
+      // pivot: largest magnitude in column p among rows >= p, smallest row on ties
+      double v = (lane >= p && lane < s) ? fabs(M[w][lane][p]) : -1.0;
+      int q = lane;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, v, off);
+        const int oq = __shfl_xor_sync(0xffffffffu, q, off);
+        if (ov > v || (ov == v && oq < q)) { v = ov; q = oq; }
+      }
+      if (q != p) {
+        for (int c = lane; c <= s; c += 32) {
+          const double tmp = M[w][p][c];
+          M[w][p][c] = M[w][q][c];
+          M[w][q][c] = tmp;
+        }
+      }
+      __syncwarp();
+      if (lane > p && lane < s) {
+        const double f = M[w][lane][p] / M[w][p][p];
+        for (int c = p + 1; c <= s; ++c) M[w][lane][c] -= f * M[w][p][c];
+      }
+      __syncwarp();
+    }
+    for (int p = s - 1; p >= 0; --p) {      // column-oriented back substitution
+      if (lane == p) zs[w][p] = M[w][p][s] / M[w][p][p];
+      __syncwarp();
+      if (lane < p) M[w][lane][s] -= M[w][lane][p] * zs[w][p];
+      __syncwarp();
+    }
+  }
+  for (int i = lane; i < n; i += 32) {
+    double v = 0.0;
+    if (used[w][i]) {
+      v = a0[i];
+      for (int c = 0; c < s; ++c) v += Nmat[(size_t)i * s + c] * zs[w][c];
+    }
+    as[w][i] = v;
+    a_out[(size_t)b * n + i] = v;
+  }
+  __syncwarp();
+  // residual max_j |sum_i a_i B[i, j] - 1| over the cyclic windows
+  double worst = 0.0;
+  for (int j = lane; j < n; j += 32) {
+    double acc = 0.0;
+    for (int t = 0; t <= s; ++t) {
+      int i = j - t;
+      if (i < 0) i += n;
+      acc += as[w][i] * coef[(size_t)i * (s + 1) + t];
+    }
+    const double r = fabs(acc - 1.0);
+    worst = fmax(worst, isnan(r) ? (double)INFINITY : r);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) worst = fmax(worst, __shfl_xor_sync(0xffffffffu, worst, off));
+  if (lane == 0) {
+    if (resid_out) resid_out[b] = worst;
+    if (maxres) atomicMax(reinterpret_cast<unsigned long long *>(maxres), (unsigned long long)__double_as_longlong(worst));
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Weighted reduction.  Each thread owns V consecutive parameters and walks the rows of the coded
+// matrix in increasing worker index (fixed order => run-to-run identical), skipping zero weights.
+// ------------------------------------------------------------------------------------------
+template <typename CT, int V>
+__global__ void __launch_bounds__(256) decode_kernel(const CT *__restrict__ coded, const double *__restrict__ a, int n,
+                                                     long long l, float *__restrict__ grad) {
+  __shared__ double as[NGC_MAX_N];
+  for (int i = threadIdx.x; i < n; i += blockDim.x) as[i] = a[i];
+  __syncthreads();
+  const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+  if (col >= l) return;
+  double acc[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) acc[e] = 0.0;
+#pragma unroll 4
+  for (int i = 0; i < n; ++i) {
+    const double ai = as[i];
+    if (ai == 0.0) continue;
+    const CT *src = coded + (size_t)i * l + col;
+    alignas(16) CT v[V];
+    if (V * sizeof(CT) == 16) *reinterpret_cast<uint4 *>(v) = __ldg(reinterpret_cast<const uint4 *>(src));
+    else if (V * sizeof(CT) == 8) *reinterpret_cast<uint2 *>(v) = __ldg(reinterpret_cast<const uint2 *>(src));
+    else v[0] = __ldg(src);
+#pragma unroll
+    for (int e = 0; e < V; ++e) acc[e] = fma(ai, (double)v[e], acc[e]);
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) grad[col + e] = (float)acc[e];
+}
+
+template <typename CT, int V>
+cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, cudaStream_t stream) {
+  const long long threads = (l + V - 1) / V;
+  const unsigned blocks = (unsigned)((threads + 255) / 256);
+  decode_kernel<CT, V><<<blocks, 256, 0, stream>>>(static_cast<const CT *>(coded), a, n, l, grad);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *masks_dev, MaskArg one, int batch,
+                                double *a_dev, double *resid_dev, double *maxres_dev, cudaStream_t stream) {
+  const ngc_level_t &lv = p.lv[layer];
+  const unsigned blocks = (unsigned)((batch + kSolveWarps - 1) / kSolveWarps);
+  decode_solve_kernel<<<blocks, kSolveWarps * 32, 0, stream>>>(masks_dev, one, batch, p.n, lv.s, lv.d_a0, lv.d_N,
+                                                              lv.d_coef, a_dev, resid_dev, maxres_dev);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
+                          cudaStream_t stream) {
+  // widest vector that keeps every row 16- / 8-byte aligned
+  if (coded_dtype == NGC_F64) {
+    if (l % 2 == 0) return run_decode<double, 2>(coded, a_dev, n, l, grad, stream);
+    return run_decode<double, 1>(coded, a_dev, n, l, grad, stream);
+  }
+  if (l % 4 == 0) return run_decode<float, 4>(coded, a_dev, n, l, grad, stream);
+  if (l % 2 == 0) return run_decode<float, 2>(coded, a_dev, n, l, grad, stream);
+  return run_decode<float, 1>(coded, a_dev, n, l, grad, stream);
+}
+
+}  // namespace ngc

@@ -1,0 +1,51 @@
+// Launchers implemented in the .cu files; called by the C-ABI entry points in ngc_api.cu.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "ngc_internal.h"
+
+namespace ngc {
+
+// How the global row range [0, T) is cut into `grid` contiguous CTA ranges and how the
+// per-CTA partial gradients of one partition group are laid out in the scratch buffer.
+struct RowSplit {
+  long long T;       // total rows = n_groups * rows_g
+  long long rows_g;  // rows per partition group (one atomic task)
+  int grid;          // CTAs; grid <= T so that no CTA range is empty
+  int P;             // scratch slots per group = max number of CTAs touching one group
+};
+
+__host__ __device__ inline long long split_begin(const RowSplit &s, long long c) { return (c * s.T) / s.grid; }
+// CTA whose range contains global row `row`.
+__host__ __device__ inline int split_owner(const RowSplit &s, long long row) {
+  return (int)(((row + 1) * s.grid - 1) / s.T);
+}
+
+RowSplit make_row_split(int n_groups, long long rows_g, int max_grid);
+
+// Streaming GEMV pair (least squares / logistic): partial gradients of every CTA range
+// into scratch `ws` laid out [group][slot][d].
+cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const void *X, const float *y,
+                             const float *theta, float *ws, int *status, cudaStream_t stream);
+
+// Sums the scratch slots of each group (fixed order) and applies the sparse code rows:
+// coded[i] = sum_t coef[i][t] * g_{(i+t) mod n}.
+cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const double *d_coef, int n, int s,
+                                  int d, void *coded, int coded_dtype, cudaStream_t stream);
+
+struct MaskArg {
+  uint64_t w[2];
+};
+// Decoding vectors: one warp per pattern.  masks_dev == nullptr -> single pattern `one`.
+cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *masks_dev, MaskArg one, int batch,
+                                double *a_dev, double *resid_dev, double *maxres_dev, cudaStream_t stream);
+
+// g = sum_i a_i coded[i], a read from device memory (zeros skipped).
+cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
+                          cudaStream_t stream);
+
+int device_sm_count();
+
+}  // namespace ngc

@@ -1,0 +1,385 @@
+// Streaming GEMV pair for the least-squares and logistic partial gradients
+// (Section II-C: g_j = sum over the rows of partition j of the per-sample loss gradient):
+//     z = X_j theta,   r = act(z) - y_j,   g_j = X_j^T r
+// fused so that every row of the data matrix is read from device memory exactly once.
+//
+// One persistent CTA per SM owns a contiguous range of the global row space.  Row tiles
+// are brought into shared memory by bulk asynchronous copies (TMA, mbarrier completion)
+// several stages ahead; every thread owns a fixed set of 16-byte column vectors, keeps
+// theta and its slice of the gradient in registers, pulls its slice of the tile into
+// registers once and uses it twice (dot product, then rank-1 update).  Row dot products
+// are reduced with warp shuffles plus one shared-memory exchange per tile.
+#include <cuda_bf16.h>
+
+#include "ngc_device.h"
+
+namespace ngc {
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxStages = 8;
+constexpr int kSmemReserve = 2048;       // barriers + reduction exchange + flags
+constexpr int kSmemMax = 232448;         // 227 KB opt-in limit per CTA
+constexpr long long kWaitCycles = 4000000000ll;
+
+struct GemvParams {
+  const unsigned char *X;
+  const float *y;
+  const float *theta;
+  float *ws;
+  int *status;
+  RowSplit split;
+  int d;
+  int row_bytes;
+  int stage_bytes;
+  int stages;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kWaitCycles SM cycles and reports failure instead of hanging.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+template <typename XT>
+struct Vec;
+template <>
+struct Vec<float> {
+  static constexpr int N = 4;
+  __device__ static __forceinline__ void unpack(const uint4 &u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y);
+    f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+  }
+};
+template <>
+struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static __forceinline__ void unpack(const uint4 &u, float (&f)[8]) {
+    f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+    f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+    f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+    f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+  }
+};
+
+// Walks the tiles of one CTA range: at most R rows, never crossing a partition-group boundary.
+struct TileWalk {
+  long long cur, end, rows_g;
+  __device__ __forceinline__ bool done() const { return cur >= end; }
+  __device__ __forceinline__ void next(int R, long long &row0, int &nrows, bool &seg_last) {
+    const long long g = cur / rows_g;
+    long long seg_end = (g + 1) * rows_g;
+    if (seg_end > end) seg_end = end;
+    long long e = cur + R;
+    if (e > seg_end) e = seg_end;
+    row0 = cur;
+    nrows = (int)(e - cur);
+    seg_last = (e == seg_end);
+    cur = e;
+  }
+};
+
+template <typename XT, int VPT, int R, int ACT>
+__global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams p) {
+  constexpr int VN = Vec<XT>::N;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char *tiles = smem;
+  unsigned char *tail = smem + (size_t)p.stages * p.stage_bytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(tail);                    // kMaxStages
+  float *red = reinterpret_cast<float *>(tail + 128);                     // [2][R][kWarps]
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + 128 + 2 * R * kWarps * 4);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nv = p.d / VN;  // 16-byte vectors per row
+
+  if (tid == 0) {
+    for (int s = 0; s < p.stages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  const long long rb = split_begin(p.split, blockIdx.x), re = split_begin(p.split, blockIdx.x + 1);
+  TileWalk prod{rb, re, p.split.rows_g}, cons{rb, re, p.split.rows_g};
+  int issued = 0;  // tiles issued by thread 0
+
+  auto issue = [&]() {
+    long long row0; int nrows; bool last;
+    prod.next(R, row0, nrows, last);
+    const int st = issued % p.stages;
+    const uint32_t bar = smem_u32(&bars[st]);
+    const uint32_t bytes = (uint32_t)nrows * (uint32_t)p.row_bytes;
+    mbar_expect_tx(bar, bytes);
+    bulk_g2s(smem_u32(tiles + (size_t)st * p.stage_bytes), p.X + (size_t)row0 * p.row_bytes, bytes, bar);
+    ++issued;
+  };
+  if (tid == 0)
+    for (int s = 0; s < p.stages - 1 && !prod.done(); ++s) issue();
+
+  // theta slice and gradient accumulators of this thread
+  float th[VPT][VN], acc[VPT][VN];
+#pragma unroll
+  for (int c = 0; c < VPT; ++c) {
+    const int v = tid + c * kThreads;
+#pragma unroll
+    for (int e = 0; e < VN; ++e) {
+      th[c][e] = (v < nv) ? __ldg(p.theta + (size_t)v * VN + e) : 0.f;
+      acc[c][e] = 0.f;
+    }
+  }
+
+  int t = 0;
+  bool failed = false;
+  while (!cons.done()) {
+    if (tid == 0 && !prod.done()) issue();  // refills the stage every thread left before the last barrier
+    long long row0; int nrows; bool seg_last;
+    cons.next(R, row0, nrows, seg_last);
+    float yv[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) yv[r] = (r < nrows) ? __ldg(p.y + row0 + r) : 0.f;
+
+    const int st = t % p.stages;
+    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)((t / p.stages) & 1))) {
+      failed = true;
+      *abort_flag = 1;
+    }
+    const unsigned char *tile = tiles + (size_t)st * p.stage_bytes;
+    uint4 xr[R][VPT];
+    float pd[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      pd[r] = 0.f;
+#pragma unroll
+      for (int c = 0; c < VPT; ++c) {
+        const int v = tid + c * kThreads;
+        if (v < nv && r < nrows)
+          xr[r][c] = *reinterpret_cast<const uint4 *>(tile + (size_t)r * p.row_bytes + (size_t)v * 16);
+        else
+          xr[r][c] = make_uint4(0u, 0u, 0u, 0u);
+        float f[VN];
+        Vec<XT>::unpack(xr[r][c], f);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) pd[r] = fmaf(f[e], th[c][e], pd[r]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) pd[r] += __shfl_xor_sync(0xffffffffu, pd[r], off);
+    }
+    float *rbuf = red + (t & 1) * (R * kWarps);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) rbuf[r * kWarps + warp] = pd[r];
+    }
+    __syncthreads();
+    if (*abort_flag) break;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float z = 0.f;
+#pragma unroll
+      for (int w4 = 0; w4 < kWarps / 4; ++w4) {
+        const float4 q = *reinterpret_cast<const float4 *>(rbuf + r * kWarps + w4 * 4);
+        z += q.x; z += q.y; z += q.z; z += q.w;
+      }
+      float res;
+      if (ACT == 1) res = 1.f / (1.f + expf(-z)) - yv[r];
+      else res = z - yv[r];
+      if (r < nrows) {
+#pragma unroll
+        for (int c = 0; c < VPT; ++c) {
+          float f[VN];
+          Vec<XT>::unpack(xr[r][c], f);
+#pragma unroll
+          for (int e = 0; e < VN; ++e) acc[c][e] = fmaf(res, f[e], acc[c][e]);
+        }
+      }
+    }
+    if (seg_last) {
+      const long long g = row0 / p.split.rows_g;
+      const int piece = (int)blockIdx.x - split_owner(p.split, g * p.split.rows_g);
+      float *dst = p.ws + ((size_t)g * p.split.P + piece) * p.d;
+#pragma unroll
+      for (int c = 0; c < VPT; ++c) {
+        const int v = tid + c * kThreads;
+        if (v < nv) {
+#pragma unroll
+          for (int e4 = 0; e4 < VN / 4; ++e4)
+            *reinterpret_cast<float4 *>(dst + (size_t)v * VN + e4 * 4) =
+                make_float4(acc[c][e4 * 4], acc[c][e4 * 4 + 1], acc[c][e4 * 4 + 2], acc[c][e4 * 4 + 3]);
+        }
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[c][e] = 0.f;
+      }
+    }
+    ++t;
+  }
+  if (failed) atomicExch(p.status, 1);
+  if (*abort_flag && tid == 0) {
+    // drain copies that are still in flight before the CTA (and its shared memory) goes away
+    for (int u = t; u < issued; ++u) mbar_wait(smem_u32(&bars[u % p.stages]), (uint32_t)((u / p.stages) & 1));
+  }
+}
+
+template <typename XT, int VPT, int R, int ACT>
+cudaError_t launch_one(const GemvParams &p, cudaStream_t stream) {
+  const size_t smem = (size_t)p.stages * p.stage_bytes + kSmemReserve;
+  auto kern = gemv_pair_kernel<XT, VPT, R, ACT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<p.split.grid, kThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename XT, int ACT>
+cudaError_t launch_shape(GemvParams &p, cudaStream_t stream) {
+  const int nv = p.d / Vec<XT>::N;
+  int vpt = (nv + kThreads - 1) / kThreads;
+  int R;
+  if (vpt <= 1) { vpt = 1; R = 8; }
+  else if (vpt == 2) { R = 4; }
+  else if (vpt <= 4) { vpt = 4; R = 2; }
+  else return cudaErrorInvalidValue;
+  p.stage_bytes = R * p.row_bytes;
+  int stages = (kSmemMax - kSmemReserve) / p.stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return cudaErrorInvalidValue;
+  p.stages = stages;
+  if (vpt == 1) return launch_one<XT, 1, 8, ACT>(p, stream);
+  if (vpt == 2) return launch_one<XT, 2, 4, ACT>(p, stream);
+  return launch_one<XT, 4, 2, ACT>(p, stream);
+}
+
+}  // namespace
+
+RowSplit make_row_split(int n_groups, long long rows_g, int max_grid) {
+  RowSplit s;
+  s.T = (long long)n_groups * rows_g;
+  s.rows_g = rows_g;
+  s.grid = (int)(s.T < max_grid ? s.T : max_grid);
+  int P = 1;
+  for (int g = 0; g < n_groups; ++g) {
+    const int c0 = split_owner(s, g * rows_g), c1 = split_owner(s, (g + 1) * rows_g - 1);
+    if (c1 - c0 + 1 > P) P = c1 - c0 + 1;
+  }
+  s.P = P;
+  return s;
+}
+
+cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const void *X, const float *y,
+                             const float *theta, float *ws, int *status, cudaStream_t stream) {
+  GemvParams p;
+  p.X = static_cast<const unsigned char *>(X);
+  p.y = y;
+  p.theta = theta;
+  p.ws = ws;
+  p.status = status;
+  p.split = split;
+  p.d = m.d;
+  const int act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
+  if (m.x_dtype == NGC_F32) {
+    p.row_bytes = m.d * 4;
+    return act ? launch_shape<float, 1>(p, stream) : launch_shape<float, 0>(p, stream);
+  }
+  p.row_bytes = m.d * 2;
+  return act ? launch_shape<__nv_bfloat16, 1>(p, stream) : launch_shape<__nv_bfloat16, 0>(p, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Combine + encode: G[j] = sum of the scratch slots of group j (fp64, fixed order), then the sparse
+// code rows x_i = sum_t B[i, i+t] g_{i+t}  (Section II-C, X = B G with the cyclic supports of Lemma 1).
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kEncCols = 128;  // columns per block
+constexpr int kEncRows = 16;   // workers per block
+
+template <typename CT>
+__global__ void __launch_bounds__(kEncCols) combine_encode_kernel(const RowSplit split, const float *__restrict__ ws,
+                                                                 const double *__restrict__ coef, int n, int s, int d,
+                                                                 CT *__restrict__ coded) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double *Gs = reinterpret_cast<double *>(smem_raw);            // [kEncRows + s][kEncCols]
+  double *cf = Gs + (size_t)(kEncRows + s) * kEncCols;          // [kEncRows][s+1]
+  const int tid = threadIdx.x;
+  const int col = blockIdx.x * kEncCols + tid;
+  const int i0 = blockIdx.y * kEncRows;
+  const int ni = min(kEncRows, n - i0);
+  for (int e = tid; e < ni * (s + 1); e += kEncCols) cf[e] = coef[(size_t)i0 * (s + 1) + e];
+  __syncthreads();
+  if (col >= d) return;
+  const int ng = min(ni + s, n);  // groups i0 .. i0+ng-1 (mod n) are needed
+  for (int u = 0; u < ng; ++u) {
+    const int g = (i0 + u) % n;
+    const int c0 = split_owner(split, (long long)g * split.rows_g);
+    const int c1 = split_owner(split, (long long)(g + 1) * split.rows_g - 1);
+    const float *src = ws + ((size_t)g * split.P) * d + col;
+    double sum = 0.0;
+    for (int pce = 0; pce <= c1 - c0; ++pce) sum += (double)src[(size_t)pce * d];
+    Gs[u * kEncCols + tid] = sum;
+  }
+  for (int ii = 0; ii < ni; ++ii) {
+    double acc = 0.0;
+    for (int t = 0; t <= s; ++t) {
+      int u = ii + t;  // slot of group (i0 + ii + t) mod n; wraps only when the block holds all n groups
+      if (ng == n && u >= n) u -= n;
+      acc = fma(cf[ii * (s + 1) + t], Gs[u * kEncCols + tid], acc);
+    }
+    coded[(size_t)(i0 + ii) * d + col] = (CT)acc;
+  }
+}
+}  // namespace
+
+cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const double *d_coef, int n, int s, int d,
+                                  void *coded, int coded_dtype, cudaStream_t stream) {
+  dim3 grid((d + kEncCols - 1) / kEncCols, (n + kEncRows - 1) / kEncRows);
+  const size_t smem = ((size_t)(kEncRows + s) * kEncCols + (size_t)kEncRows * (s + 1)) * sizeof(double);
+  if (coded_dtype == NGC_F64) {
+    cudaError_t e = cudaFuncSetAttribute(combine_encode_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    combine_encode_kernel<double><<<grid, kEncCols, smem, stream>>>(split, ws, d_coef, n, s, d,
+                                                                    static_cast<double *>(coded));
+  } else {
+    cudaError_t e = cudaFuncSetAttribute(combine_encode_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    combine_encode_kernel<float><<<grid, kEncCols, smem, stream>>>(split, ws, d_coef, n, s, d,
+                                                                   static_cast<float *>(coded));
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace ngc

@@ -1,0 +1,48 @@
+"""Full-size workloads in the launch configuration the benchmark times, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import ngc_inputs
+import paper_2212_08580_b200 as ngc
+from oracle import ngc_oracle as orc
+from tests._util import coded_torch_dtype, model_of, oracle_G, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,tol", [("logistic20", 1e-5), ("lsq100", 1e-5)])
+def test_full_size_step_matches_oracle(name, tol):
+    w = ngc_inputs.WORKLOADS[name]
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    pl = orc.plan(w.n, list(w.levels), w.seed)
+    l = w.n_params
+    cdt = p.coded_dtype(m)
+    coded = torch.empty((w.n, l), dtype=coded_torch_dtype(cdt), device="cuda")
+    grad = torch.empty(l, dtype=torch.float32, device="cuda")
+    G = oracle_G(w, X, y, theta)                     # every partition, fp64, from the same bits
+    g_full = G.sum(axis=0)
+    done = 0
+    for it in range(12):
+        t = ngc_inputs.pattern_times(w, it)
+        want = orc.select(t, list(w.levels), 0.0, 0.0)
+        if want is None:
+            with pytest.raises(ngc.NgcError):
+                p.step(m, theta, X, y, t, coded, grad)
+            continue
+        info = p.step(m, theta, X, y, t, coded, grad)
+        torch.cuda.synchronize()
+        assert info.layer == want["level"] and np.array_equal(info.responsive(), want["S"])
+        assert info.latency == want["latency"]
+        B = pl["B"][info.layer]
+        if done < 2:                                  # coded rows, sampled
+            got = coded.cpu().numpy()
+            want_coded = orc.encode(B, G)
+            for i in (0, w.n // 2, w.n - 1):
+                assert rel_l2(got[i], want_coded[i]) < tol
+        assert rel_l2(grad.cpu().numpy(), g_full) < tol
+        done += 1
+    assert done >= 8
+    assert p.device_status() < 1e-6
