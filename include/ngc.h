@@ -187,6 +187,15 @@ int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta
 int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate, double p_fail,
                      double *task_times_host);
 
+/*
+ * Timing of the dominant kernel of ngc_grad_encode (the fused gradient kernel).  While enabled,
+ * every ngc_grad_encode call brackets that kernel with CUDA events on the launching stream.
+ * ngc_profile_read synchronises those events, returns their summed elapsed milliseconds and the
+ * number of bracketed launches since the last read, and resets both.
+ */
+int ngc_profile_enable(ngc_plan_t *plan, int on);
+int ngc_profile_read(ngc_plan_t *plan, double *ms_total_out, int64_t *launches_out);
+
 /* Bytes of device workspace the plan currently holds. */
 size_t ngc_workspace_bytes(const ngc_plan_t *plan);
 /* Synchronises the device and returns NGC_OK or NGC_ERR_TIMEOUT / NGC_ERR_SINGULAR from the status

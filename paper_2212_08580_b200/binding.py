@@ -75,6 +75,8 @@ def load_library() -> C.CDLL:
         "ngc_step": (i32, [vp, P(Model), vp, vp, vp, P(dbl), vp, vp, P(StepInfo), vp]),
         "ngc_step_host": (i32, [vp, P(Model), vp, vp, vp, P(dbl), vp, P(StepInfo)]),
         "ngc_sample_times": (i32, [u64, i32, i32, dbl, dbl, dbl, P(dbl)]),
+        "ngc_profile_enable": (i32, [vp, i32]),
+        "ngc_profile_read": (i32, [vp, P(dbl), P(i64)]),
         "ngc_workspace_bytes": (C.c_size_t, [vp]),
         "ngc_device_status": (i32, [vp, P(dbl)]),
         "ngc_last_cuda_error": (i32, [vp]),
@@ -227,6 +229,15 @@ class Plan:
         res = C.c_double()
         self._check(self._lib.ngc_device_status(self._h, C.byref(res)), "ngc_device_status")
         return res.value
+
+    def profile_enable(self, on: bool):
+        self._check(self._lib.ngc_profile_enable(self._h, int(on)), "ngc_profile_enable")
+
+    def profile_read(self):
+        """(summed milliseconds of the bracketed fused-gradient kernels, their count) since the last read."""
+        ms, cnt = C.c_double(), C.c_int64()
+        self._check(self._lib.ngc_profile_read(self._h, C.byref(ms), C.byref(cnt)), "ngc_profile_read")
+        return ms.value, cnt.value
 
     def workspace_bytes(self) -> int:
         return int(self._lib.ngc_workspace_bytes(self._h))

@@ -114,6 +114,18 @@ int check_model(const ngc_plan_s *p, const ngc_model_t *m) {
   return NGC_OK;
 }
 
+// Records one event of a begin/end pair on `stream` when profiling is on.
+int profile_mark(ngc_plan_s *p, cudaStream_t stream) {
+  if (!p->profiling) return NGC_OK;
+  if (p->ev_used == p->ev.size()) {
+    cudaEvent_t e;
+    NGC_CUDA(p, cudaEventCreate(&e));
+    p->ev.push_back(e);
+  }
+  NGC_CUDA(p, cudaEventRecord(static_cast<cudaEvent_t>(p->ev[p->ev_used++]), stream));
+  return NGC_OK;
+}
+
 // The residual |a B - 1| above which a decode is reported as NGC_ERR_SINGULAR.
 constexpr double kResidualLimit = 1e-6;
 
@@ -142,6 +154,7 @@ void ngc_plan_destroy(ngc_plan_t *p) {
     cudaFree(p->st_coded);
     cudaFree(p->st_grad);
   }
+  for (void *e : p->ev) cudaEventDestroy(static_cast<cudaEvent_t>(e));
   delete p;
 }
 
@@ -165,8 +178,10 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     const ngc::RowSplit split = ngc::make_row_split(p->n, (long long)p->q * m->rows_per_partition, sms);
     rc = ensure_ws(p, (size_t)p->n * split.P * m->d * sizeof(float));
     if (rc != NGC_OK) return rc;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     NGC_CUDA(p, ngc::launch_gemv_pair(*m, split, X, static_cast<const float *>(y), static_cast<const float *>(theta),
                                       static_cast<float *>(p->ws), p->d_status, stream));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     NGC_CUDA(p, ngc::launch_combine_encode(split, static_cast<const float *>(p->ws), lv.d_coef, p->n, lv.s, m->d,
                                            coded, cdt, stream));
     p->launches += 2;
@@ -281,6 +296,28 @@ int ngc_device_status(ngc_plan_t *p, double *residual_out) {
   if (residual_out) *residual_out = mr;
   if (st[0] != 0) return NGC_ERR_TIMEOUT;
   if (!(mr <= kResidualLimit)) return NGC_ERR_SINGULAR;
+  return NGC_OK;
+}
+
+int ngc_profile_enable(ngc_plan_t *p, int on) {
+  if (!p) return NGC_ERR_INVALID;
+  p->profiling = on != 0;
+  return NGC_OK;
+}
+
+int ngc_profile_read(ngc_plan_t *p, double *ms_total, int64_t *launches) {
+  if (!p || !ms_total || !launches) return NGC_ERR_INVALID;
+  *ms_total = 0.0;
+  *launches = 0;
+  for (size_t i = 0; i + 1 < p->ev_used; i += 2) {
+    cudaEvent_t a = static_cast<cudaEvent_t>(p->ev[i]), b = static_cast<cudaEvent_t>(p->ev[i + 1]);
+    NGC_CUDA(p, cudaEventSynchronize(b));
+    float ms = 0.f;
+    NGC_CUDA(p, cudaEventElapsedTime(&ms, a, b));
+    *ms_total += ms;
+    *launches += 1;
+  }
+  p->ev_used = 0;
   return NGC_OK;
 }
 

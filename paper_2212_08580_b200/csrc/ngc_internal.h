@@ -39,6 +39,10 @@ struct ngc_plan_s {
   // staging for ngc_step_host
   void *st_X = nullptr, *st_y = nullptr, *st_theta = nullptr, *st_coded = nullptr, *st_grad = nullptr;
   size_t st_X_bytes = 0, st_y_bytes = 0, st_theta_bytes = 0, st_coded_bytes = 0, st_grad_bytes = 0;
+  // optional event brackets around the dominant kernel
+  bool profiling = false;
+  std::vector<void *> ev;      // cudaEvent_t pairs, reused
+  size_t ev_used = 0;
   int last_cuda = 0;
   int64_t launches = 0;
 };
