@@ -73,53 +73,116 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                : "memory");
 }
 
+// Two fp32 values in one 64-bit register pair, the operand type of the packed FMA.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// d = a * b + d on both halves (one issue slot for two fused multiply-adds).
+__device__ __forceinline__ void fma2(f32x2 &d, f32x2 a, f32x2 b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
 template <typename XT>
 struct Vec;
 template <>
 struct Vec<float> {
-  static constexpr int N = 4;
-  __device__ static __forceinline__ void unpack(const uint4 &u, float (&f)[4]) {
-    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y);
-    f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+  static constexpr int N = 4;  // elements per 16-byte vector
+  __device__ static __forceinline__ void unpack(const uint4 &u, f32x2 (&f)[2]) {
+    f[0] = pack2(__uint_as_float(u.x), __uint_as_float(u.y));
+    f[1] = pack2(__uint_as_float(u.z), __uint_as_float(u.w));
   }
 };
 template <>
 struct Vec<__nv_bfloat16> {
   static constexpr int N = 8;
-  __device__ static __forceinline__ void unpack(const uint4 &u, float (&f)[8]) {
-    f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
-    f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
-    f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
-    f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+  __device__ static __forceinline__ void unpack(const uint4 &u, f32x2 (&f)[4]) {
+    f[0] = pack2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+    f[1] = pack2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+    f[2] = pack2(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+    f[3] = pack2(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
   }
 };
 
 // Walks the tiles of one CTA range: at most R rows, never crossing a partition-group boundary.
 struct TileWalk {
-  long long cur, end, rows_g;
-  __device__ __forceinline__ bool done() const { return cur >= end; }
-  __device__ __forceinline__ void next(int R, long long &row0, int &nrows, bool &seg_last) {
-    const long long g = cur / rows_g;
-    long long seg_end = (g + 1) * rows_g;
+  long long cur, end, seg_end, rows_g;
+  int group;
+  __device__ __forceinline__ void init(long long b, long long e, long long rg) {
+    cur = b; end = e; rows_g = rg;
+    group = (int)(b / rg);
+    seg_end = (long long)(group + 1) * rg;
     if (seg_end > end) seg_end = end;
+  }
+  __device__ __forceinline__ bool done() const { return cur >= end; }
+  // returns the tile starting at `cur`; seg_last = it closes this CTA's piece of partition group `g`
+  __device__ __forceinline__ void next(int R, long long &row0, int &nrows, bool &seg_last, int &g) {
     long long e = cur + R;
     if (e > seg_end) e = seg_end;
     row0 = cur;
     nrows = (int)(e - cur);
+    g = group;
     seg_last = (e == seg_end);
     cur = e;
+    if (seg_last) {
+      ++group;
+      seg_end += rows_g;
+      if (seg_end > end) seg_end = end;
+    }
   }
 };
+
+// Sum over the 32 lanes of R per-lane values with R/2 + ... + 1 + log2(32/R) shuffles: at each of the
+// first log2(R) steps a lane hands half of its values to its partner and keeps the other half.
+// Afterwards lane l holds the full sum of row  bitrev-free index  (l >> (5 - log2 R)).
+template <int R>
+__device__ __forceinline__ float warp_reduce_rows(float (&v)[R], int lane) {
+  int width = 16;
+#pragma unroll
+  for (int n = R; n > 1; n >>= 1) {
+    const bool upper = (lane & width) != 0;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const float send = upper ? v[i] : v[i + n / 2];
+      const float keep = upper ? v[i + n / 2] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, width);
+    }
+    width >>= 1;
+  }
+  float x = v[0];
+#pragma unroll
+  for (; width > 0; width >>= 1) x += __shfl_xor_sync(0xffffffffu, x, width);
+  return x;
+}
+
+template <int R>
+struct Log2;
+template <> struct Log2<2> { static constexpr int v = 1; };
+template <> struct Log2<4> { static constexpr int v = 2; };
+template <> struct Log2<8> { static constexpr int v = 3; };
 
 template <typename XT, int VPT, int R, int ACT>
 __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams p) {
   constexpr int VN = Vec<XT>::N;
+  constexpr int VH = VN / 2;  // packed pairs per vector
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *tiles = smem;
   unsigned char *tail = smem + (size_t)p.stages * p.stage_bytes;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(tail);                    // kMaxStages
-  float *red = reinterpret_cast<float *>(tail + 128);                     // [2][R][kWarps]
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + 128 + 2 * R * kWarps * 4);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(tail);        // kMaxStages
+  float *red = reinterpret_cast<float *>(tail + 128);         // [R][kWarps] per-warp partial dot products
+  float *resv = red + R * kWarps;                             // [R] residuals of the tile's rows
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(resv + R);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nv = p.d / VN;  // 16-byte vectors per row
@@ -133,119 +196,134 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
   __syncthreads();
 
   const long long rb = split_begin(p.split, blockIdx.x), re = split_begin(p.split, blockIdx.x + 1);
-  TileWalk prod{rb, re, p.split.rows_g}, cons{rb, re, p.split.rows_g};
-  int issued = 0;  // tiles issued by thread 0
+  TileWalk prod, cons;
+  prod.init(rb, re, p.split.rows_g);
+  cons.init(rb, re, p.split.rows_g);
+  int issued = 0;        // tiles issued by thread 0
+  int issue_stage = 0;
 
   auto issue = [&]() {
-    long long row0; int nrows; bool last;
-    prod.next(R, row0, nrows, last);
-    const int st = issued % p.stages;
-    const uint32_t bar = smem_u32(&bars[st]);
+    long long row0; int nrows, g; bool last;
+    prod.next(R, row0, nrows, last, g);
+    const uint32_t bar = smem_u32(&bars[issue_stage]);
     const uint32_t bytes = (uint32_t)nrows * (uint32_t)p.row_bytes;
     mbar_expect_tx(bar, bytes);
-    bulk_g2s(smem_u32(tiles + (size_t)st * p.stage_bytes), p.X + (size_t)row0 * p.row_bytes, bytes, bar);
+    bulk_g2s(smem_u32(tiles + (size_t)issue_stage * p.stage_bytes), p.X + (size_t)row0 * p.row_bytes, bytes, bar);
     ++issued;
+    if (++issue_stage == p.stages) issue_stage = 0;
   };
   if (tid == 0)
     for (int s = 0; s < p.stages - 1 && !prod.done(); ++s) issue();
 
-  // theta slice and gradient accumulators of this thread
-  float th[VPT][VN], acc[VPT][VN];
+  // theta slice and gradient accumulators of this thread, as packed pairs
+  f32x2 th[VPT][VH], acc[VPT][VH];
+  bool vok[VPT];
 #pragma unroll
   for (int c = 0; c < VPT; ++c) {
     const int v = tid + c * kThreads;
+    vok[c] = v < nv;
 #pragma unroll
-    for (int e = 0; e < VN; ++e) {
-      th[c][e] = (v < nv) ? __ldg(p.theta + (size_t)v * VN + e) : 0.f;
-      acc[c][e] = 0.f;
+    for (int e = 0; e < VH; ++e) {
+      const float2 t2 = vok[c] ? __ldg(reinterpret_cast<const float2 *>(p.theta) + (size_t)v * VH + e)
+                               : make_float2(0.f, 0.f);
+      th[c][e] = pack2(t2.x, t2.y);
+      acc[c][e] = pack2(0.f, 0.f);
     }
   }
 
-  int t = 0;
+  const uint32_t tiles_u32 = smem_u32(tiles) + (uint32_t)tid * 16u;
+  int t = 0, st = 0;
+  uint32_t parity = 0;
   bool failed = false;
   while (!cons.done()) {
     if (tid == 0 && !prod.done()) issue();  // refills the stage every thread left before the last barrier
-    long long row0; int nrows; bool seg_last;
-    cons.next(R, row0, nrows, seg_last);
-    float yv[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) yv[r] = (r < nrows) ? __ldg(p.y + row0 + r) : 0.f;
+    long long row0; int nrows, g; bool seg_last;
+    cons.next(R, row0, nrows, seg_last, g);
+    // the warps that will finish the row sums fetch the labels early
+    float yrow = 0.f;
+    if (warp < R && lane == 0 && warp < nrows) yrow = __ldg(p.y + row0 + warp);
 
-    const int st = t % p.stages;
-    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)((t / p.stages) & 1))) {
+    if (!mbar_wait(smem_u32(&bars[st]), parity)) {
       failed = true;
       *abort_flag = 1;
     }
-    const unsigned char *tile = tiles + (size_t)st * p.stage_bytes;
+    const uint32_t tile = tiles_u32 + (uint32_t)st * (uint32_t)p.stage_bytes;
     uint4 xr[R][VPT];
     float pd[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      pd[r] = 0.f;
+      f32x2 d2 = pack2(0.f, 0.f);
 #pragma unroll
       for (int c = 0; c < VPT; ++c) {
-        const int v = tid + c * kThreads;
-        if (v < nv && r < nrows)
-          xr[r][c] = *reinterpret_cast<const uint4 *>(tile + (size_t)r * p.row_bytes + (size_t)v * 16);
+        if (vok[c] && r < nrows)
+          xr[r][c] = lds128(tile + (uint32_t)r * (uint32_t)p.row_bytes + (uint32_t)c * (kThreads * 16));
         else
           xr[r][c] = make_uint4(0u, 0u, 0u, 0u);
-        float f[VN];
+        f32x2 f[VH];
         Vec<XT>::unpack(xr[r][c], f);
 #pragma unroll
-        for (int e = 0; e < VN; ++e) pd[r] = fmaf(f[e], th[c][e], pd[r]);
+        for (int e = 0; e < VH; ++e) fma2(d2, f[e], th[c][e]);
       }
+      float lo, hi;
+      unpack2(d2, lo, hi);
+      pd[r] = lo + hi;
     }
+    const float rowsum = warp_reduce_rows<R>(pd, lane);
+    if ((lane & (31 >> Log2<R>::v)) == 0) red[(lane >> (5 - Log2<R>::v)) * kWarps + warp] = rowsum;
+    __syncthreads();
+    if (warp < R) {  // warp r finishes row r: sum over the kWarps partials, then the residual
+      float z = (lane < kWarps) ? red[warp * kWarps + lane] : 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) pd[r] += __shfl_xor_sync(0xffffffffu, pd[r], off);
-    }
-    float *rbuf = red + (t & 1) * (R * kWarps);
-    if (lane == 0) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) rbuf[r * kWarps + warp] = pd[r];
+      for (int off = kWarps / 2; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+      if (lane == 0) {
+        float res;
+        if (ACT == 1) res = 1.f / (1.f + expf(-z)) - yrow;
+        else res = z - yrow;
+        resv[warp] = (warp < nrows) ? res : 0.f;
+      }
     }
     __syncthreads();
     if (*abort_flag) break;
+    if (sizeof(XT) == 2) {
+      // keep the packed words, not their unpacked copies, live across the barriers
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < VPT; ++c)
+          asm volatile("" : "+r"(xr[r][c].x), "+r"(xr[r][c].y), "+r"(xr[r][c].z), "+r"(xr[r][c].w));
+    }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      float z = 0.f;
+      const float res = resv[r];
+      const f32x2 res2 = pack2(res, res);
 #pragma unroll
-      for (int w4 = 0; w4 < kWarps / 4; ++w4) {
-        const float4 q = *reinterpret_cast<const float4 *>(rbuf + r * kWarps + w4 * 4);
-        z += q.x; z += q.y; z += q.z; z += q.w;
-      }
-      float res;
-      if (ACT == 1) res = 1.f / (1.f + expf(-z)) - yv[r];
-      else res = z - yv[r];
-      if (r < nrows) {
+      for (int c = 0; c < VPT; ++c) {
+        f32x2 f[VH];
+        Vec<XT>::unpack(xr[r][c], f);
 #pragma unroll
-        for (int c = 0; c < VPT; ++c) {
-          float f[VN];
-          Vec<XT>::unpack(xr[r][c], f);
-#pragma unroll
-          for (int e = 0; e < VN; ++e) acc[c][e] = fmaf(res, f[e], acc[c][e]);
-        }
+        for (int e = 0; e < VH; ++e) fma2(acc[c][e], res2, f[e]);
       }
     }
     if (seg_last) {
-      const long long g = row0 / p.split.rows_g;
-      const int piece = (int)blockIdx.x - split_owner(p.split, g * p.split.rows_g);
-      float *dst = p.ws + ((size_t)g * p.split.P + piece) * p.d;
+      const int piece = (int)blockIdx.x - split_owner(p.split, (long long)g * p.split.rows_g);
+      float *dst = p.ws + ((size_t)g * p.split.P + piece) * p.d + (size_t)tid * VN;
 #pragma unroll
       for (int c = 0; c < VPT; ++c) {
-        const int v = tid + c * kThreads;
-        if (v < nv) {
+        if (vok[c]) {
 #pragma unroll
-          for (int e4 = 0; e4 < VN / 4; ++e4)
-            *reinterpret_cast<float4 *>(dst + (size_t)v * VN + e4 * 4) =
-                make_float4(acc[c][e4 * 4], acc[c][e4 * 4 + 1], acc[c][e4 * 4 + 2], acc[c][e4 * 4 + 3]);
+          for (int e = 0; e < VH; e += 2) {
+            float4 o;
+            unpack2(acc[c][e], o.x, o.y);
+            unpack2(acc[c][e + 1], o.z, o.w);
+            *reinterpret_cast<float4 *>(dst + (size_t)c * (kThreads * VN) + e * 2) = o;
+          }
         }
 #pragma unroll
-        for (int e = 0; e < VN; ++e) acc[c][e] = 0.f;
+        for (int e = 0; e < VH; ++e) acc[c][e] = pack2(0.f, 0.f);
       }
     }
     ++t;
+    if (++st == p.stages) { st = 0; parity ^= 1u; }
   }
   if (failed) atomicExch(p.status, 1);
   if (*abort_flag && tid == 0) {
