@@ -47,7 +47,8 @@ enum {
   NGC_ERR_SINGULAR = -3,    /* decoding vector residual |a B - 1| above threshold */
   NGC_ERR_CUDA = -4,        /* a CUDA runtime call failed; see ngc_last_cuda_error */
   NGC_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reported by ngc_device_status) */
-  NGC_ERR_NOMEM = -6        /* host allocation failed */
+  NGC_ERR_NOMEM = -6,       /* host allocation failed */
+  NGC_ERR_TOO_LARGE = -7    /* problem needs more scratch than the fixed array of ngc_grad_encode_static holds */
 };
 
 typedef enum { NGC_LSQ = 0, NGC_LOGISTIC = 1, NGC_SOFTMAX = 2, NGC_MLP = 3 } ngc_model_kind;
@@ -186,6 +187,35 @@ int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta
  */
 int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate, double p_fail,
                      double *task_times_host);
+
+/*
+ * Variant of ngc_grad_encode (least squares and logistic only) that allocates NO device memory.
+ * (The paper has no counterpart: this is a property of the library, not of the method.)
+ *
+ * It is meant for callers that cannot call cudaMalloc at this point of their program: a process
+ * whose GPU memory has been handed over completely to its own pool allocator, so that a raw
+ * allocation would fail or fragment that pool, or a latency-critical loop that cannot take the
+ * device-wide stall an allocation or a free may cause.  The scratch that ngc_grad_encode takes
+ * from the plan (per-CTA partial gradients, a device copy of the component code's coefficients, a
+ * status word) lives instead in one fixed array of NGC_STATIC_SCRATCH_BYTES inside the library
+ * image; every GPU that loads the library holds that much until the process exits.
+ *
+ * Arguments are those of ngc_grad_encode; the plan is only read (its host tables), so a plan that
+ * has never touched the GPU works.  status_dev may be NULL; if given, it points to one int32 in
+ * device memory that is cleared by the call and set to 1 if a bounded device-side wait gave up.
+ * Limit: n * slots * d * 4 bytes of partial gradients must fit in 8 MiB, where slots is the largest
+ * number of CTAs that share one partition group (about 148 / n + 2 on a B200); larger problems are
+ * refused with NGC_ERR_TOO_LARGE before anything is enqueued.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before any stream capture begins.  All calls, from every plan and stream,
+ * share the one array: two calls that overlap on the GPU race on it, so keep them ordered.  The
+ * array keeps the previous call's contents; the call clears the status word itself and writes
+ * every scratch slot before reading it.
+ */
+#define NGC_STATIC_SCRATCH_BYTES (256 + NGC_MAX_N * (NGC_MAX_S + 1) * 8 + 8 * 1024 * 1024)
+int ngc_grad_encode_static(const ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev,
+                           const void *X_dev, const void *y_dev, int layer, void *coded_dev,
+                           int32_t *status_dev, void *cuda_stream);
 
 /*
  * Timing of the dominant kernel of ngc_grad_encode (the fused gradient kernel).  While enabled,

@@ -69,6 +69,7 @@ def load_library() -> C.CDLL:
         "ngc_coded_dtype": (i32, [vp, P(Model)]),
         "ngc_select": (i32, [vp, P(dbl), P(StepInfo)]),
         "ngc_grad_encode": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp]),
+        "ngc_grad_encode_static": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp, vp]),
         "ngc_decode_vector": (i32, [vp, i32, P(C.c_int32), i32, P(dbl)]),
         "ngc_decode_vectors": (i32, [vp, i32, P(C.c_int32), i32, i32, P(dbl), P(dbl)]),
         "ngc_decode": (i32, [vp, i32, P(C.c_int32), i32, vp, i32, i64, vp, vp]),
@@ -190,6 +191,13 @@ class Plan:
     def grad_encode(self, model: Model, theta, X, y, layer: int, coded, stream: int = 0):
         self._check(self._lib.ngc_grad_encode(self._h, C.byref(model), _addr(theta), _addr(X), _addr(y), layer,
                                               _addr(coded), stream), "ngc_grad_encode")
+
+    def grad_encode_static(self, model: Model, theta, X, y, layer: int, coded, status=None, stream: int = 0):
+        """ngc_grad_encode_static: same result as grad_encode, but no device memory is allocated
+        (scratch comes from a fixed array inside the library; see include/ngc.h for the limit)."""
+        self._check(self._lib.ngc_grad_encode_static(self._h, C.byref(model), _addr(theta), _addr(X), _addr(y), layer,
+                                                     _addr(coded), _addr(status) if status is not None else None,
+                                                     stream), "ngc_grad_encode_static")
 
     def decode_vector(self, layer: int, S) -> np.ndarray:
         S = np.ascontiguousarray(S, dtype=np.int32)

@@ -338,6 +338,7 @@ const char *ngc_strerror(int status) {
     case NGC_ERR_CUDA: return "CUDA runtime error";
     case NGC_ERR_TIMEOUT: return "bounded device-side wait gave up";
     case NGC_ERR_NOMEM: return "out of host memory";
+    case NGC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of ngc_grad_encode_static";
     default: return "unknown status";
   }
 }
