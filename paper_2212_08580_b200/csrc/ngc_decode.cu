@@ -113,41 +113,57 @@ decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, 
 }
 
 // ------------------------------------------------------------------------------------------
-// Weighted reduction.  Each thread owns V consecutive parameters and walks the rows of the coded
-// matrix in increasing worker index (fixed order => run-to-run identical), skipping zero weights.
+// Weighted reduction.  A block owns 32*V consecutive parameters; its 8 warps take the rows of the
+// coded matrix round-robin (lane = V consecutive parameters, 16-byte loads), zero weights skipped,
+// and the 8 partial sums are added in warp order, so reruns give identical bits.
 // ------------------------------------------------------------------------------------------
+constexpr int kDecWarps = 8;
+
 template <typename CT, int V>
-__global__ void __launch_bounds__(256) decode_kernel(const CT *__restrict__ coded, const double *__restrict__ a, int n,
-                                                     long long l, float *__restrict__ grad) {
+__global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
+                                                              int n, long long l, float *__restrict__ grad) {
   __shared__ double as[NGC_MAX_N];
+  __shared__ double part[kDecWarps][32 * V];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int i = threadIdx.x; i < n; i += blockDim.x) as[i] = a[i];
   __syncthreads();
-  const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
-  if (col >= l) return;
+  const long long col = ((long long)blockIdx.x * 32 + lane) * V;
   double acc[V];
 #pragma unroll
   for (int e = 0; e < V; ++e) acc[e] = 0.0;
+  if (col < l) {
 #pragma unroll 4
-  for (int i = 0; i < n; ++i) {
-    const double ai = as[i];
-    if (ai == 0.0) continue;
-    const CT *src = coded + (size_t)i * l + col;
-    alignas(16) CT v[V];
-    if (V * sizeof(CT) == 16) *reinterpret_cast<uint4 *>(v) = __ldg(reinterpret_cast<const uint4 *>(src));
-    else if (V * sizeof(CT) == 8) *reinterpret_cast<uint2 *>(v) = __ldg(reinterpret_cast<const uint2 *>(src));
-    else v[0] = __ldg(src);
+    for (int i = warp; i < n; i += kDecWarps) {
+      const double ai = as[i];
+      if (ai == 0.0) continue;
+      const CT *src = coded + (size_t)i * l + col;
+      alignas(16) CT v[V];
+      if (V * sizeof(CT) == 16) *reinterpret_cast<uint4 *>(v) = __ldg(reinterpret_cast<const uint4 *>(src));
+      else if (V * sizeof(CT) == 8) *reinterpret_cast<uint2 *>(v) = __ldg(reinterpret_cast<const uint2 *>(src));
+      else v[0] = __ldg(src);
 #pragma unroll
-    for (int e = 0; e < V; ++e) acc[e] = fma(ai, (double)v[e], acc[e]);
+      for (int e = 0; e < V; ++e) acc[e] = fma(ai, (double)v[e], acc[e]);
+    }
   }
 #pragma unroll
-  for (int e = 0; e < V; ++e) grad[col + e] = (float)acc[e];
+  for (int e = 0; e < V; ++e) part[warp][lane * V + e] = acc[e];
+  __syncthreads();
+  for (int c = threadIdx.x; c < 32 * V; c += blockDim.x) {
+    const long long gc = (long long)blockIdx.x * 32 * V + c;
+    if (gc < l) {
+      double sum = 0.0;
+#pragma unroll
+      for (int w = 0; w < kDecWarps; ++w) sum += part[w][c];
+      grad[gc] = (float)sum;
+    }
+  }
 }
 
 template <typename CT, int V>
 cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, cudaStream_t stream) {
-  const long long threads = (l + V - 1) / V;
-  const unsigned blocks = (unsigned)((threads + 255) / 256);
-  decode_kernel<CT, V><<<blocks, 256, 0, stream>>>(static_cast<const CT *>(coded), a, n, l, grad);
+  const long long per_block = 32 * V;
+  const unsigned blocks = (unsigned)((l + per_block - 1) / per_block);
+  decode_kernel<CT, V><<<blocks, kDecWarps * 32, 0, stream>>>(static_cast<const CT *>(coded), a, n, l, grad);
   return cudaGetLastError();
 }
 

@@ -399,63 +399,76 @@ cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const 
 // ---------------------------------------------------------------------------------------------
 // Combine + encode: G[j] = sum of the scratch slots of group j (fp64, fixed order), then the sparse
 // code rows x_i = sum_t B[i, i+t] g_{i+t}  (Section II-C, X = B G with the cyclic supports of Lemma 1).
+// A block owns 128 columns x 8 workers; its 8 warps split the group sums and then the workers, each
+// lane carrying 4 consecutive columns (16-byte loads of the fp32 partials).
 // ---------------------------------------------------------------------------------------------
 namespace {
 constexpr int kEncCols = 128;  // columns per block
-constexpr int kEncRows = 16;   // workers per block
+constexpr int kEncRows = 8;    // workers per block
+constexpr int kEncWarps = 8;
 
 template <typename CT>
-__global__ void __launch_bounds__(kEncCols) combine_encode_kernel(const RowSplit split, const float *__restrict__ ws,
-                                                                 const double *__restrict__ coef, int n, int s, int d,
-                                                                 CT *__restrict__ coded) {
+__global__ void __launch_bounds__(kEncWarps * 32)
+combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const double *__restrict__ coef, int n, int s,
+                      int d, CT *__restrict__ coded) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double *Gs = reinterpret_cast<double *>(smem_raw);            // [kEncRows + s][kEncCols]
   double *cf = Gs + (size_t)(kEncRows + s) * kEncCols;          // [kEncRows][s+1]
-  const int tid = threadIdx.x;
-  const int col = blockIdx.x * kEncCols + tid;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int col = blockIdx.x * kEncCols + lane * 4;
   const int i0 = blockIdx.y * kEncRows;
   const int ni = min(kEncRows, n - i0);
-  for (int e = tid; e < ni * (s + 1); e += kEncCols) cf[e] = coef[(size_t)i0 * (s + 1) + e];
+  for (int e = tid; e < ni * (s + 1); e += kEncWarps * 32) cf[e] = coef[(size_t)i0 * (s + 1) + e];
+  const int ng = min(ni + s, n);  // groups i0 .. i0+ng-1 (mod n) are needed
+  if (col < d) {
+    for (int u = warp; u < ng; u += kEncWarps) {
+      const int g = (i0 + u) % n;
+      const int c0 = split_owner(split, (long long)g * split.rows_g);
+      const int c1 = split_owner(split, (long long)(g + 1) * split.rows_g - 1);
+      const float *src = ws + ((size_t)g * split.P) * d + col;
+      double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 4
+      for (int pce = 0; pce <= c1 - c0; ++pce) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(src + (size_t)pce * d));
+        s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+      }
+      double *dst = Gs + u * kEncCols + lane * 4;
+      dst[0] = s0; dst[1] = s1; dst[2] = s2; dst[3] = s3;
+    }
+  }
   __syncthreads();
   if (col >= d) return;
-  const int ng = min(ni + s, n);  // groups i0 .. i0+ng-1 (mod n) are needed
-  for (int u = 0; u < ng; ++u) {
-    const int g = (i0 + u) % n;
-    const int c0 = split_owner(split, (long long)g * split.rows_g);
-    const int c1 = split_owner(split, (long long)(g + 1) * split.rows_g - 1);
-    const float *src = ws + ((size_t)g * split.P) * d + col;
-    double sum = 0.0;
-    for (int pce = 0; pce <= c1 - c0; ++pce) sum += (double)src[(size_t)pce * d];
-    Gs[u * kEncCols + tid] = sum;
-  }
-  for (int ii = 0; ii < ni; ++ii) {
-    double acc = 0.0;
+  for (int ii = warp; ii < ni; ii += kEncWarps) {
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
     for (int t = 0; t <= s; ++t) {
       int u = ii + t;  // slot of group (i0 + ii + t) mod n; wraps only when the block holds all n groups
       if (ng == n && u >= n) u -= n;
-      acc = fma(cf[ii * (s + 1) + t], Gs[u * kEncCols + tid], acc);
+      const double c = cf[ii * (s + 1) + t];
+      const double *gsrc = Gs + u * kEncCols + lane * 4;
+      a0 = fma(c, gsrc[0], a0); a1 = fma(c, gsrc[1], a1); a2 = fma(c, gsrc[2], a2); a3 = fma(c, gsrc[3], a3);
     }
-    coded[(size_t)(i0 + ii) * d + col] = (CT)acc;
+    CT *dst = coded + (size_t)(i0 + ii) * d + col;
+    if (sizeof(CT) == 8) {
+      reinterpret_cast<double2 *>(dst)[0] = make_double2(a0, a1);
+      reinterpret_cast<double2 *>(dst)[1] = make_double2(a2, a3);
+    } else {
+      *reinterpret_cast<float4 *>(dst) = make_float4((float)a0, (float)a1, (float)a2, (float)a3);
+    }
   }
 }
 }  // namespace
 
 cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const double *d_coef, int n, int s, int d,
                                   void *coded, int coded_dtype, cudaStream_t stream) {
+  if (d % 4 != 0) return cudaErrorInvalidValue;
   dim3 grid((d + kEncCols - 1) / kEncCols, (n + kEncRows - 1) / kEncRows);
   const size_t smem = ((size_t)(kEncRows + s) * kEncCols + (size_t)kEncRows * (s + 1)) * sizeof(double);
   if (coded_dtype == NGC_F64) {
-    cudaError_t e = cudaFuncSetAttribute(combine_encode_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    combine_encode_kernel<double><<<grid, kEncCols, smem, stream>>>(split, ws, d_coef, n, s, d,
-                                                                    static_cast<double *>(coded));
+    combine_encode_kernel<double><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
+                                                                          static_cast<double *>(coded));
   } else {
-    cudaError_t e = cudaFuncSetAttribute(combine_encode_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    combine_encode_kernel<float><<<grid, kEncCols, smem, stream>>>(split, ws, d_coef, n, s, d,
-                                                                   static_cast<float *>(coded));
+    combine_encode_kernel<float><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
+                                                                         static_cast<float *>(coded));
   }
   return cudaGetLastError();
 }
