@@ -187,7 +187,27 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     p->launches += 2;
     return NGC_OK;
   }
-  return NGC_ERR_INVALID;  // softmax / MLP paths are not built yet
+  if (m->kind == NGC_SOFTMAX) {
+    if (m->x_dtype != NGC_BF16 || m->n_classes % 16 != 0 || m->n_classes < 16 || m->n_classes > 256 || m->d % 8 != 0)
+      return NGC_ERR_INVALID;
+    const int sms = ngc::device_sm_count();
+    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
+    rc = ensure_ws(p, ngc::softmax_scratch_bytes(p->k, m->rows_per_partition, m->d, m->n_classes));
+    if (rc != NGC_OK) return rc;
+    float *G = nullptr;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_softmax_grad(p->k, m->rows_per_partition, m->d, m->n_classes, X, static_cast<const int *>(y),
+                                         static_cast<const float *>(theta), static_cast<unsigned char *>(p->ws), &G,
+                                         p->d_status, sms, stream));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    // G is [n][q][l]: group g of q consecutive partitions, one scratch slot per partition
+    ngc::RowSplit split;
+    split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
+    NGC_CUDA(p, ngc::launch_combine_encode(split, G, lv.d_coef, p->n, lv.s, (int)ngc_num_params(m), coded, cdt, stream));
+    p->launches += 4;
+    return NGC_OK;
+  }
+  return NGC_ERR_INVALID;  // the MLP path is not built yet
 }
 
 int ngc_decode_vectors(ngc_plan_t *p, int layer, const int32_t *S, int nS, int batch, double *a_out,

@@ -46,6 +46,11 @@ cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *
 cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
                           cudaStream_t stream);
 
+// Softmax-regression partial gradients on the tensor cores (X bf16): G[k][d*C] fp32 inside `scratch`.
+size_t softmax_scratch_bytes(int k, int rows, int d, int C);
+cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, const int *y, const float *W,
+                                unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream);
+
 int device_sm_count();
 
 }  // namespace ngc
