@@ -404,16 +404,16 @@ cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const 
 // ---------------------------------------------------------------------------------------------
 namespace {
 constexpr int kEncCols = 128;  // columns per block
-constexpr int kEncRows = 8;    // workers per block
 constexpr int kEncWarps = 8;
 
 template <typename CT>
 __global__ void __launch_bounds__(kEncWarps * 32)
 combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const double *__restrict__ coef, int n, int s,
-                      int d, CT *__restrict__ coded) {
+                      int d, CT *__restrict__ coded, int kEncRows /* workers per block */) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double *Gs = reinterpret_cast<double *>(smem_raw);            // [kEncRows + s][kEncCols]
-  double *cf = Gs + (size_t)(kEncRows + s) * kEncCols;          // [kEncRows][s+1]
+  const int held = min(kEncRows + s, n);
+  double *Gs = reinterpret_cast<double *>(smem_raw);            // [held][kEncCols]
+  double *cf = Gs + (size_t)held * kEncCols;                    // [kEncRows][s+1]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int col = blockIdx.x * kEncCols + lane * 4;
   const int i0 = blockIdx.y * kEncRows;
@@ -461,14 +461,24 @@ combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const 
 cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const double *d_coef, int n, int s, int d,
                                   void *coded, int coded_dtype, cudaStream_t stream) {
   if (d % 4 != 0) return cudaErrorInvalidValue;
-  dim3 grid((d + kEncCols - 1) / kEncCols, (n + kEncRows - 1) / kEncRows);
-  const size_t smem = ((size_t)(kEncRows + s) * kEncCols + (size_t)kEncRows * (s + 1)) * sizeof(double);
+  // Few column tiles (small models): 8 workers per block for parallelism, at the price of re-reading
+  // (8+s)/8 of the group sums.  Many column tiles: one block takes all n workers and reads everything once.
+  const int col_tiles = (d + kEncCols - 1) / kEncCols;
+  const int enc_rows = (col_tiles >= 4 * device_sm_count()) ? n : 8;
+  dim3 grid(col_tiles, (n + enc_rows - 1) / enc_rows);
+  const int held = (enc_rows + s < n) ? enc_rows + s : n;
+  const size_t smem = ((size_t)held * kEncCols + (size_t)enc_rows * (s + 1)) * sizeof(double);
+  cudaError_t e;
   if (coded_dtype == NGC_F64) {
+    e = cudaFuncSetAttribute(combine_encode_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     combine_encode_kernel<double><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
-                                                                          static_cast<double *>(coded));
+                                                                          static_cast<double *>(coded), enc_rows);
   } else {
+    e = cudaFuncSetAttribute(combine_encode_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     combine_encode_kernel<float><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
-                                                                         static_cast<float *>(coded));
+                                                                         static_cast<float *>(coded), enc_rows);
   }
   return cudaGetLastError();
 }

@@ -11,7 +11,7 @@ from tests._util import coded_torch_dtype, model_of, oracle_G, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,tol", [("logistic20", 1e-5), ("lsq100", 1e-5)])
+@pytest.mark.parametrize("name,tol", [("logistic20", 1e-5), ("lsq100", 1e-5), ("softmax50", 1e-2)])
 def test_full_size_step_matches_oracle(name, tol):
     w = ngc_inputs.WORKLOADS[name]
     X, y, theta = ngc_inputs.make_data(w, "cuda")
