@@ -269,11 +269,14 @@ def mlp_unpack(theta, d, hidden, n_classes):
     return W1, b1, W2, b2
 
 
-def grad_mlp(X, labels, theta, hidden, n_classes):
+def grad_mlp(X, labels, theta, hidden, n_classes, relu_mask=None):
     """One-hidden-layer ReLU network with softmax cross-entropy, back-propagated.
 
     Parameters flattened as [W1 (d x hidden, row-major), b1, W2 (hidden x C), b2];
-    ReLU'(0) = 0.
+    ReLU'(0) = 0.  `relu_mask` (rows x hidden, 0/1), when given, replaces the
+    derivative decision pre > 0: that decision is an integer taken from floating
+    point, and a checker may want both sides to take it in the same precision.
+    Everything else stays fp64.
     """
     X = np.asarray(X, dtype=np.float64)
     d = X.shape[1]
@@ -284,7 +287,7 @@ def grad_mlp(X, labels, theta, hidden, n_classes):
     P[np.arange(X.shape[0]), np.asarray(labels)] -= 1.0      # delta2
     dW2 = h.T @ P
     db2 = P.sum(axis=0)
-    delta1 = (P @ W2.T) * (pre > 0.0)
+    delta1 = (P @ W2.T) * ((pre > 0.0) if relu_mask is None else np.asarray(relu_mask, dtype=np.float64))
     dW1 = X.T @ delta1
     db1 = delta1.sum(axis=0)
     return np.concatenate([dW1.reshape(-1), db1, dW2.reshape(-1), db2])

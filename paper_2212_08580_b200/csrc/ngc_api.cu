@@ -203,11 +203,34 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     // G is [n][q][l]: group g of q consecutive partitions, one scratch slot per partition
     ngc::RowSplit split;
     split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
-    NGC_CUDA(p, ngc::launch_combine_encode(split, G, lv.d_coef, p->n, lv.s, (int)ngc_num_params(m), coded, cdt, stream));
+    const long long l = ngc_num_params(m);
+    NGC_CUDA(p, ngc::launch_encode_long(split, G, l, lv.d_coef, p->n, lv.s, l, coded, cdt, stream));
     p->launches += 4;
     return NGC_OK;
   }
-  return NGC_ERR_INVALID;  // the MLP path is not built yet
+  if (m->kind == NGC_MLP) {
+    if (m->x_dtype != NGC_F32) return NGC_ERR_INVALID;
+    const int h = m->hidden, C = m->n_classes;
+    if (m->d % 8 != 0 || h % 16 != 0 || h < 16 || h > 512 || (h > 256 && h % 256 != 0) || C < 1 || C > 16)
+      return NGC_ERR_INVALID;
+    const int sms = ngc::device_sm_count();
+    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
+    rc = ensure_ws(p, ngc::mlp_scratch_bytes(p->k, m->rows_per_partition, m->d, h, C));
+    if (rc != NGC_OK) return rc;
+    float *G = nullptr;
+    long long ldG = 0;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_mlp_grad(p->k, m->rows_per_partition, m->d, h, C, static_cast<const float *>(X),
+                                     static_cast<const int *>(y), static_cast<const float *>(theta),
+                                     static_cast<unsigned char *>(p->ws), &G, &ldG, p->d_status, sms, stream));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    ngc::RowSplit split;
+    split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
+    NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, ngc_num_params(m), coded, cdt, stream));
+    p->launches += 6;
+    return NGC_OK;
+  }
+  return NGC_ERR_INVALID;
 }
 
 int ngc_decode_vectors(ngc_plan_t *p, int layer, const int32_t *S, int nS, int batch, double *a_out,

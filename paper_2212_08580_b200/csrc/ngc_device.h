@@ -46,6 +46,18 @@ cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *
 cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
                           cudaStream_t stream);
 
+// Same encode for long gradients (dense models): every partial gradient is read once, windows live in
+// registers.  ws is [group][slot][ld_ws] fp32, ld_ws a multiple of 4 and >= d.
+cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
+                               int s, long long d, void *coded, int coded_dtype, cudaStream_t stream);
+
+// MLP (one hidden ReLU layer, softmax cross-entropy) partial gradients on the tensor cores (X fp32):
+// G[k][*G_ld] fp32 inside `scratch`, each row holding [dW1, db1, dW2, db2].
+size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C);
+cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
+                            unsigned char *scratch, float **G_out, long long *G_ld, int *status, int sms,
+                            cudaStream_t stream);
+
 // Softmax-regression partial gradients on the tensor cores (X bf16): G[k][d*C] fp32 inside `scratch`.
 size_t softmax_scratch_bytes(int k, int rows, int d, int C);
 cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, const int *y, const float *W,
