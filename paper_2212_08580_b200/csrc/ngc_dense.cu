@@ -28,16 +28,17 @@ constexpr int kTcThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr int kSmemTc = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 
-struct TcParams {
-  int k;       // partitions
-  int rows;    // rows per partition
-  int d;       // features
-  int C;       // classes (multiple of 16, <= 256)
-  int tiles_per_part;
-  int num_tiles;
-  int num_k;   // K chunks of 64
-  const int *y;
-  __nv_bfloat16 *R;   // [k][rows][C]
+// Forward contraction D[128 rows x N] = X_tile[128 x K] * B^T with a fused epilogue.
+// Tile = (partition j, block of 128 rows, block nt of 256 output columns).
+struct FwdParams {
+  int rows;       // rows per partition
+  int n_total;    // output columns in all (classes, or hidden units)
+  int row_blocks, n_tiles, num_tiles;
+  int num_k;      // K chunks of 64
+  const int *y;   // class labels (softmax epilogue)
+  __nv_bfloat16 *out;  // [k][rows][out_ld]
+  int out_ld;
+  int ones_col;   // relu epilogue: column that receives 1.0 (followed by 7 zeros); -1 = none
   int *status;
 };
 
@@ -170,10 +171,12 @@ __global__ void convert_x_kernel(const float *__restrict__ X, __nv_bfloat16 *__r
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward: tile = (partition j, block of 128 rows).  D[128 x C] = X_tile[128 x d] * W[d x C].
+// Forward contractions.  EPI = 0: softmax residual  R = softmax(Z) - onehot(y)  (needs all classes in one
+// tile).  EPI = 1: H = relu(Z) (first MLP layer; bias already folded into the contraction).
 // ------------------------------------------------------------------------------------------------
+template <int EPI>
 __global__ void __launch_bounds__(kTcThreads, 1)
-softmax_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const TcParams p) {
+fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ unsigned char smem_raw[];
   const Smem s = carve(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -185,23 +188,24 @@ softmax_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       int st = 0;
       uint32_t ph = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        const int j = tile / p.tiles_per_part, rb = tile % p.tiles_per_part;
+        const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
           mbar_expect_tx(s.full[st], kStageBytes);
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
           tma_load_3d(a, &tmX, kc * 64, rb * 128, j, s.full[st]);
-          tma_load_2d(a + kABytes, &tmW, kc * 64, 0, s.full[st]);
+          tma_load_2d(a + kABytes, &tmW, kc * 64, nt * 256, s.full[st]);
           if (++st == kStages) { st = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = instr_desc_bf16(128, p.C, 0, 0);
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
+        const int nt = tile % p.n_tiles;
+        const uint32_t idesc = instr_desc_bf16(128, min(256, p.n_total - nt * 256), 0, 0);
         if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
         tc_fence_after();
         const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
@@ -227,45 +231,66 @@ softmax_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     int buf = 0;
     uint32_t aph = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      const int j = tile / p.tiles_per_part, rb = tile % p.tiles_per_part;
+      const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
       if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
       tc_fence_after();
       const int row = rb * 128 + q * 32 + lane;
       const bool valid = row < p.rows;
+      const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
-      const int label = valid ? p.y[(size_t)j * p.rows + row] : -1;
+      const int ncol = min(256, p.n_total - nt * 256);
+      __nv_bfloat16 *dst = p.out + grow * p.out_ld + nt * 256;
       float v[32];
-      float mx = -INFINITY;
-      for (int c0 = 0; c0 < p.C; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
+      if (EPI == 0) {
+        const int label = valid ? p.y[grow] : -1;
+        float mx = -INFINITY;
+        for (int c0 = 0; c0 < ncol; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (c0 + i < p.C) mx = fmaxf(mx, v[i]);
-      }
-      float sum = 0.f;
-      for (int c0 = 0; c0 < p.C; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (c0 + i < p.C) sum += __expf(v[i] - mx);
-      }
-      const float inv = 1.f / sum;
-      __nv_bfloat16 *dst = p.R + ((size_t)j * p.rows + (valid ? row : 0)) * p.C;
-      for (int c0 = 0; c0 < p.C; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
-#pragma unroll
-        for (int g8 = 0; g8 < 4; ++g8) {
-          uint32_t w[4];
-#pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            const int c = c0 + g8 * 8 + h * 2;
-            const float r0 = __expf(v[g8 * 8 + h * 2] - mx) * inv - (c == label ? 1.f : 0.f);
-            const float r1 = __expf(v[g8 * 8 + h * 2 + 1] - mx) * inv - (c + 1 == label ? 1.f : 0.f);
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
-            w[h] = *reinterpret_cast<const uint32_t *>(&b2);
-          }
-          if (valid && c0 + g8 * 8 < p.C) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i < ncol) mx = fmaxf(mx, v[i]);
         }
+        float sum = 0.f;
+        for (int c0 = 0; c0 < ncol; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i < ncol) sum += __expf(v[i] - mx);
+        }
+        const float inv = 1.f / sum;
+        for (int c0 = 0; c0 < ncol; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const int c = c0 + g8 * 8 + h * 2;
+              const float r0 = __expf(v[g8 * 8 + h * 2] - mx) * inv - (c == label ? 1.f : 0.f);
+              const float r1 = __expf(v[g8 * 8 + h * 2 + 1] - mx) * inv - (c + 1 == label ? 1.f : 0.f);
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
+              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+            }
+            if (valid && c0 + g8 * 8 < ncol) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      } else {
+        for (int c0 = 0; c0 < ncol; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const __nv_bfloat162 b2 =
+                  __floats2bfloat162_rn(fmaxf(v[g8 * 8 + h * 2], 0.f), fmaxf(v[g8 * 8 + h * 2 + 1], 0.f));
+              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+            }
+            if (valid && c0 + g8 * 8 < ncol) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        if (valid && nt == 0 && p.ones_col >= 0)  // bf16 1.0 followed by zeros
+          *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
       }
       tc_fence_before();
       mbar_arrive(s.tempty[buf]);
@@ -274,6 +299,138 @@ softmax_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
   }
   epilogue_teardown(s, warp, tmem_base, failed, p.status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// MLP head on the CUDA cores (the output layer is 10-wide: no tensor-core shape):
+//   z = h W2 + b2,  delta2 = softmax(z) - onehot(y),  delta1 = (delta2 W2^T) * (h > 0).
+// h comes as bf16 rows (the forward's output); delta1 is stored as bf16 rows, delta2 as bf16 rows of 64
+// (16 used).  A block stages 64 consecutive rows of h in shared memory with coalesced loads; four
+// threads share a row (a quarter of the hidden units each), exchange their partial logits through
+// shared memory, overwrite h by delta1 in place, and the block copies the tile out coalesced.  W2 sits in
+// shared memory, padded to CPAD classes, and is read by broadcast.
+// ------------------------------------------------------------------------------------------------
+constexpr int kHeadRows = 64;
+constexpr int kHeadThreads = 256;
+
+template <int CPAD>
+__global__ void __launch_bounds__(kHeadThreads)
+mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C, const float *__restrict__ W2,
+                const float *__restrict__ b2, const int *__restrict__ y, long long rows_total,
+                __nv_bfloat16 *__restrict__ D1, __nv_bfloat16 *__restrict__ D2) {
+  extern __shared__ __align__(16) unsigned char head_smem[];
+  float *w2s = reinterpret_cast<float *>(head_smem);                 // [hidden][CPAD], then b2[CPAD]
+  float *zpart = w2s + (size_t)hidden * CPAD + CPAD;                 // [4][kHeadRows][CPAD]
+  uint4 *tile = reinterpret_cast<uint4 *>(zpart + 4 * kHeadRows * CPAD);  // [kHeadRows][hpad / 8]
+  const int tid = threadIdx.x;
+  for (int e = tid; e < hidden * CPAD; e += kHeadThreads) {
+    const int hc = e / CPAD, c = e % CPAD;
+    w2s[e] = c < C ? W2[(size_t)hc * C + c] : 0.f;
+  }
+  if (tid < CPAD) w2s[hidden * CPAD + tid] = tid < C ? b2[tid] : 0.f;
+  const long long row0 = (long long)blockIdx.x * kHeadRows;
+  const int nrows = (int)min((long long)kHeadRows, rows_total - row0);
+  const int gpr = hpad / 8, hg = hidden / 8;  // 16-byte groups per stored row / per row of hidden units
+  {
+    const uint4 *src = reinterpret_cast<const uint4 *>(H + row0 * hpad);
+    for (int e = tid; e < nrows * gpr; e += kHeadThreads) tile[e] = __ldg(src + e);
+  }
+  __syncthreads();
+  const int part = tid >> 6, r = tid & 63;
+  const int gper = (hg + 3) / 4, g_begin = part * gper, g_end = min(hg, g_begin + gper);
+  const bool valid = r < nrows;
+  float z[CPAD];
+#pragma unroll
+  for (int c = 0; c < CPAD; ++c) z[c] = 0.f;
+  if (valid) {
+    for (int g8 = g_begin; g8 < g_end; ++g8) {
+      const uint4 u = tile[r * gpr + g8];
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float h = __uint_as_float((i & 1) ? (w[i >> 1] & 0xffff0000u) : (w[i >> 1] << 16));
+        const float4 *w2 = reinterpret_cast<const float4 *>(w2s + (size_t)(g8 * 8 + i) * CPAD);
+#pragma unroll
+        for (int c4 = 0; c4 < CPAD / 4; ++c4) {
+          const float4 ww = w2[c4];
+          z[c4 * 4] = fmaf(h, ww.x, z[c4 * 4]);
+          z[c4 * 4 + 1] = fmaf(h, ww.y, z[c4 * 4 + 1]);
+          z[c4 * 4 + 2] = fmaf(h, ww.z, z[c4 * 4 + 2]);
+          z[c4 * 4 + 3] = fmaf(h, ww.w, z[c4 * 4 + 3]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < CPAD; ++c) zpart[(part * kHeadRows + r) * CPAD + c] = z[c];
+  __syncthreads();
+  float dl[CPAD];
+  {
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < CPAD; ++c) {
+      z[c] = zpart[r * CPAD + c] + zpart[(kHeadRows + r) * CPAD + c] + zpart[(2 * kHeadRows + r) * CPAD + c] +
+             zpart[(3 * kHeadRows + r) * CPAD + c] + w2s[hidden * CPAD + c];
+      if (c < C) mx = fmaxf(mx, z[c]);
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < CPAD; ++c) {
+      dl[c] = c < C ? __expf(z[c] - mx) : 0.f;
+      sum += dl[c];
+    }
+    const float inv = 1.f / sum;
+    const int label = valid ? y[row0 + r] : -1;
+#pragma unroll
+    for (int c = 0; c < CPAD; ++c) dl[c] = c < C ? dl[c] * inv - (c == label ? 1.f : 0.f) : 0.f;
+  }
+  if (valid && part == 0) {
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float lo = 2 * i < CPAD ? dl[2 * i < CPAD ? 2 * i : 0] : 0.f;
+      const float hi = 2 * i + 1 < CPAD ? dl[2 * i + 1 < CPAD ? 2 * i + 1 : 0] : 0.f;
+      const __nv_bfloat162 b2v = __floats2bfloat162_rn(lo, hi);
+      w[i] = *reinterpret_cast<const uint32_t *>(&b2v);
+    }
+    uint4 *d2 = reinterpret_cast<uint4 *>(D2 + (row0 + r) * 64);
+    d2[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    d2[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  }
+  if (valid) {
+    for (int g8 = g_begin; g8 < g_end; ++g8) {
+      const uint4 u = tile[r * gpr + g8];
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int hh = 0; hh < 4; ++hh) {
+        float dv[2];
+#pragma unroll
+        for (int uu = 0; uu < 2; ++uu) {
+          const uint32_t bits = uu ? (w[hh] & 0xffff0000u) : (w[hh] << 16);
+          const float4 *w2 = reinterpret_cast<const float4 *>(w2s + (size_t)(g8 * 8 + hh * 2 + uu) * CPAD);
+          float acc = 0.f;
+#pragma unroll
+          for (int c4 = 0; c4 < CPAD / 4; ++c4) {
+            const float4 ww = w2[c4];
+            acc = fmaf(dl[c4 * 4], ww.x, acc);
+            acc = fmaf(dl[c4 * 4 + 1], ww.y, acc);
+            acc = fmaf(dl[c4 * 4 + 2], ww.z, acc);
+            acc = fmaf(dl[c4 * 4 + 3], ww.w, acc);
+          }
+          dv[uu] = __uint_as_float(bits) > 0.f ? acc : 0.f;
+        }
+        const __nv_bfloat162 db = __floats2bfloat162_rn(dv[0], dv[1]);
+        o[hh] = *reinterpret_cast<const uint32_t *>(&db);
+      }
+      tile[r * gpr + g8] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+  __syncthreads();
+  {
+    uint4 *dst = reinterpret_cast<uint4 *>(D1 + row0 * hidden);
+    for (int e = tid; e < nrows * hg; e += kHeadThreads) dst[e] = tile[(e / hg) * gpr + (e % hg)];
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -372,246 +529,6 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ------------------------------------------------------------------------------------------------
-// MLP forward: tile = (partition j, block of 128 rows).  pre[128 x hidden] = [X 1][W1; b1] in tensor
-// memory (up to two 256-column accumulators), then on the CUDA cores, one thread per (row, half of the
-// hidden units): h = relu(pre), z = h W2 + b2, delta2 = softmax(z) - onehot(y),
-// delta1 = (delta2 W2^T) * (pre > 0).  Stored for the backward contractions: H = [h 1] and delta1 as
-// bf16 row-major, delta2 as bf16 rows of 64 (16 used).
-// ------------------------------------------------------------------------------------------------
-constexpr int kMlpStages = 2;
-constexpr int kMlpBBytes = 512 * 64 * 2;  // 64 KB: up to 512 hidden units x 64 bf16
-constexpr int kMlpStageBytes = kABytes + kMlpBBytes;
-constexpr int kMlpThreads = 320;          // producer, MMA, 8 epilogue warps
-
-struct MlpParams {
-  int k, rows, d, hidden, C;
-  int hpad;      // row stride of H = hidden + 1 rounded up to 8
-  int tiles_per_part, num_tiles, num_k;
-  const int *y;
-  const float *W2;   // [hidden][C]
-  const float *b2;   // [C]
-  __nv_bfloat16 *H;  // [k][rows][hpad]
-  __nv_bfloat16 *D1; // [k][rows][hidden]
-  __nv_bfloat16 *D2; // [k][rows][64]
-  int *status;
-};
-
-template <int CPAD>
-__global__ void __launch_bounds__(kMlpThreads, 1)
-mlp_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const MlpParams p) {
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t base = smem_u32(smem_raw);
-  unsigned char *tiles = smem_raw + ((1024u - (base & 1023u)) & 1023u);
-  uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + kMlpStages * kMlpStageBytes);
-  uint32_t full[kMlpStages], empty[kMlpStages];
-#pragma unroll
-  for (int i = 0; i < kMlpStages; ++i) {
-    full[i] = smem_u32(&bars[i]);
-    empty[i] = smem_u32(&bars[kMlpStages + i]);
-  }
-  const uint32_t tfull = smem_u32(&bars[2 * kMlpStages]), tempty = smem_u32(&bars[2 * kMlpStages + 1]);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kMlpStages + 2]);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-  float *W2s = reinterpret_cast<float *>(tiles + kMlpStages * kMlpStageBytes + 128);  // [hidden][CPAD]
-  float *b2s = W2s + 512 * CPAD;                                                      // [CPAD]
-  float *zpart = b2s + 16;                                                            // [2][128][CPAD]
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < kMlpStages; ++i) {
-      mbar_init(full[i], 1);
-      mbar_init(empty[i], 1);
-    }
-    mbar_init(tfull, 1);
-    mbar_init(tempty, 256);
-    *abort_flag = 0;
-    mbar_fence_init();
-  }
-  for (int e = threadIdx.x; e < p.hidden * CPAD; e += kMlpThreads) {
-    const int hc = e / CPAD, c = e % CPAD;
-    W2s[e] = c < p.C ? p.W2[(size_t)hc * p.C + c] : 0.f;
-  }
-  if (threadIdx.x < CPAD) b2s[threadIdx.x] = threadIdx.x < p.C ? p.b2[threadIdx.x] : 0.f;
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  bool failed = false;
-  const int n_halves = (p.hidden + 255) / 256;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      int st = 0;
-      uint32_t ph = 0;
-      const uint32_t tx = (uint32_t)kABytes + (uint32_t)n_halves * 32768u;
-      for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        const int j = tile / p.tiles_per_part, rb = tile % p.tiles_per_part;
-        for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(empty[st], ph ^ 1u)) { failed = true; break; }
-          mbar_expect_tx(full[st], tx);
-          const uint32_t a = smem_u32(tiles + st * kMlpStageBytes);
-          tma_load_3d(a, &tmX, kc * 64, rb * 128, j, full[st]);
-          for (int h = 0; h < n_halves; ++h) tma_load_2d(a + kABytes + h * 32768, &tmW, kc * 64, h * 256, full[st]);
-          if (++st == kMlpStages) { st = 0; ph ^= 1u; }
-        }
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      int st = 0;
-      uint32_t ph = 0, aph = 0;
-      for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        if (!mbar_wait(tempty, aph ^ 1u)) { failed = true; break; }
-        tc_fence_after();
-        for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(full[st], ph)) { failed = true; break; }
-          tc_fence_after();
-          const uint32_t a = smem_u32(tiles + st * kMlpStageBytes);
-          const uint64_t ad = smem_desc_sw128(a, 16, 1024);
-          for (int h = 0; h < n_halves; ++h) {
-            const int nh = min(256, p.hidden - h * 256);
-            const uint32_t idesc = instr_desc_bf16(128, nh, 0, 0);
-            const uint64_t bd = smem_desc_sw128(a + kABytes + h * 32768, 16, 1024);
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
-              mma_bf16(tmem_base + (uint32_t)h * 256u, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc,
-                       (kc | k4) != 0);
-          }
-          mma_commit(empty[st]);
-          if (++st == kMlpStages) { st = 0; ph ^= 1u; }
-        }
-        if (failed) break;
-        mma_commit(tfull);
-        aph ^= 1u;
-      }
-    }
-  } else {
-    const int q = warp & 3;           // tensor-memory quadrant of this warp
-    const int hf = (warp - 2) >> 2;   // which 256 hidden units
-    const int rt = q * 32 + lane;     // row within the tile
-    const int h_begin = hf * 256, h_count = max(0, min(256, p.hidden - h_begin));
-    uint32_t aph = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      const int j = tile / p.tiles_per_part, rb = tile % p.tiles_per_part;
-      if (!mbar_wait(tfull, aph)) { failed = true; break; }
-      tc_fence_after();
-      const int row = rb * 128 + rt;
-      const bool valid = row < p.rows;
-      const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)h_begin;
-      const int label = valid ? p.y[grow] : -1;
-      float v[32];
-      float z[CPAD];
-#pragma unroll
-      for (int c = 0; c < CPAD; ++c) z[c] = 0.f;
-      for (int c0 = 0; c0 < h_count; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (c0 + i < h_count) {
-            const float h = fmaxf(v[i], 0.f);
-            const float4 *w2 = reinterpret_cast<const float4 *>(W2s + (size_t)(h_begin + c0 + i) * CPAD);
-#pragma unroll
-            for (int c4 = 0; c4 < CPAD / 4; ++c4) {
-              const float4 ww = w2[c4];
-              z[c4 * 4] = fmaf(h, ww.x, z[c4 * 4]);
-              z[c4 * 4 + 1] = fmaf(h, ww.y, z[c4 * 4 + 1]);
-              z[c4 * 4 + 2] = fmaf(h, ww.z, z[c4 * 4 + 2]);
-              z[c4 * 4 + 3] = fmaf(h, ww.w, z[c4 * 4 + 3]);
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int c = 0; c < CPAD; ++c) zpart[(hf * 128 + rt) * CPAD + c] = z[c];
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      float dl[CPAD];
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < CPAD; ++c) {
-        z[c] = zpart[rt * CPAD + c] + zpart[(128 + rt) * CPAD + c] + b2s[c];
-        if (c < p.C) mx = fmaxf(mx, z[c]);
-      }
-      float sum = 0.f;
-#pragma unroll
-      for (int c = 0; c < CPAD; ++c) {
-        dl[c] = c < p.C ? __expf(z[c] - mx) : 0.f;
-        sum += dl[c];
-      }
-      const float inv = 1.f / sum;
-#pragma unroll
-      for (int c = 0; c < CPAD; ++c) dl[c] = c < p.C ? dl[c] * inv - (c == label ? 1.f : 0.f) : 0.f;
-      if (hf == 0 && valid) {
-        uint32_t w[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float lo = 2 * i < CPAD ? dl[2 * i < CPAD ? 2 * i : 0] : 0.f;
-          const float hi = 2 * i + 1 < CPAD ? dl[2 * i + 1 < CPAD ? 2 * i + 1 : 0] : 0.f;
-          const __nv_bfloat162 b2v = __floats2bfloat162_rn(lo, hi);
-          w[i] = *reinterpret_cast<const uint32_t *>(&b2v);
-        }
-        uint4 *d2 = reinterpret_cast<uint4 *>(p.D2 + grow * 64);
-        d2[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        d2[1] = make_uint4(w[4], w[5], w[6], w[7]);
-        // column of ones (and padding) behind the hidden activations
-        *reinterpret_cast<uint4 *>(p.H + grow * p.hpad + p.hidden) = make_uint4(0x00003f80u, 0u, 0u, 0u);
-      }
-      __nv_bfloat16 *hrow = p.H + grow * p.hpad + h_begin;
-      __nv_bfloat16 *drow = p.D1 + grow * p.hidden + h_begin;
-      for (int c0 = 0; c0 < h_count; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
-#pragma unroll
-        for (int g8 = 0; g8 < 4; ++g8) {
-          uint32_t hw[4], dw[4];
-#pragma unroll
-          for (int hh = 0; hh < 4; ++hh) {
-            float hv[2], dv[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int i = g8 * 8 + hh * 2 + u;
-              const float pre = v[i];
-              const bool act = pre > 0.f && (c0 + i < h_count);
-              const int hc = min(h_begin + c0 + i, p.hidden - 1);
-              const float4 *w2 = reinterpret_cast<const float4 *>(W2s + (size_t)hc * CPAD);
-              float acc = 0.f;
-#pragma unroll
-              for (int c4 = 0; c4 < CPAD / 4; ++c4) {
-                const float4 ww = w2[c4];
-                acc = fmaf(dl[c4 * 4], ww.x, acc);
-                acc = fmaf(dl[c4 * 4 + 1], ww.y, acc);
-                acc = fmaf(dl[c4 * 4 + 2], ww.z, acc);
-                acc = fmaf(dl[c4 * 4 + 3], ww.w, acc);
-              }
-              hv[u] = act ? pre : 0.f;
-              dv[u] = act ? acc : 0.f;
-            }
-            const __nv_bfloat162 hb = __floats2bfloat162_rn(hv[0], hv[1]);
-            const __nv_bfloat162 db = __floats2bfloat162_rn(dv[0], dv[1]);
-            hw[hh] = *reinterpret_cast<const uint32_t *>(&hb);
-            dw[hh] = *reinterpret_cast<const uint32_t *>(&db);
-          }
-          if (valid && c0 + g8 * 8 < h_count) {
-            *reinterpret_cast<uint4 *>(hrow + c0 + g8 * 8) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-            *reinterpret_cast<uint4 *>(drow + c0 + g8 * 8) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
-          }
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(tempty);
-      aph ^= 1u;
-    }
-  }
-  if (failed) {
-    *abort_flag = 1;
-    atomicExch(p.status, 1);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
-}
-
-// ------------------------------------------------------------------------------------------------
 // Host side: tensor maps
 // ------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -685,19 +602,16 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
-  TcParams p;
-  p.k = k; p.rows = rows; p.d = d; p.C = C;
-  p.y = y; p.R = R; p.status = status;
-
-  e = cudaFuncSetAttribute(softmax_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
+  e = cudaFuncSetAttribute(fwd_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
 
-  p.tiles_per_part = (rows + 127) / 128;
-  p.num_tiles = k * p.tiles_per_part;
-  p.num_k = (d + 63) / 64;
-  softmax_fwd_kernel<<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
+  FwdParams p;
+  p.rows = rows; p.n_total = C; p.row_blocks = (rows + 127) / 128; p.n_tiles = 1;
+  p.num_tiles = k * p.row_blocks; p.num_k = (d + 63) / 64;
+  p.y = y; p.out = R; p.out_ld = C; p.ones_col = -1; p.status = status;
+  fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
@@ -711,7 +625,6 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmR, t);
   return cudaGetLastError();
 }
-
 
 namespace {
 inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
@@ -766,30 +679,36 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   transpose_to_bf16_kernel<<<tg, tb, 0, stream>>>(W1, b1, W1t, d, hidden, dpad);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-  MlpParams p;
-  p.k = k; p.rows = rows; p.d = d; p.hidden = hidden; p.C = C; p.hpad = hpad;
-  p.tiles_per_part = (rows + 127) / 128;
-  p.num_tiles = k * p.tiles_per_part;
-  p.num_k = (dpad + 63) / 64;
-  p.y = y; p.W2 = W2; p.b2 = b2; p.H = H; p.D1 = D1; p.D2 = D2; p.status = status;
-  const int cpad = (C + 3) / 4 * 4;
-  const int smem = kMlpStages * kMlpStageBytes + 1024 + 128 + (512 * cpad + 16 + 2 * 128 * cpad) * 4;
-  const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-#define NGC_LAUNCH_MLP(CP)                                                                                   \
-  do {                                                                                                       \
-    e = cudaFuncSetAttribute(mlp_fwd_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);         \
-    if (e != cudaSuccess) return e;                                                                          \
-    mlp_fwd_kernel<CP><<<grid, kMlpThreads, smem, stream>>>(tmXa, tmW, p);                                    \
-  } while (0)
-  if (cpad == 4) NGC_LAUNCH_MLP(4);
-  else if (cpad == 8) NGC_LAUNCH_MLP(8);
-  else if (cpad == 12) NGC_LAUNCH_MLP(12);
-  else NGC_LAUNCH_MLP(16);
-#undef NGC_LAUNCH_MLP
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-
+  e = cudaFuncSetAttribute(fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
+  if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
+
+  // H = relu([X 1] [W1; b1]), with its own column of ones behind the hidden units
+  FwdParams p;
+  p.rows = rows; p.n_total = hidden; p.row_blocks = (rows + 127) / 128; p.n_tiles = (hidden + 255) / 256;
+  p.num_tiles = k * p.row_blocks * p.n_tiles; p.num_k = (dpad + 63) / 64;
+  p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = hidden; p.status = status;
+  fwd_kernel<1><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+  const int cpad = (C + 3) / 4 * 4;
+  const size_t head_smem = ((size_t)hidden * cpad + cpad + 4 * kHeadRows * cpad) * sizeof(float) + (size_t)kHeadRows * hpad * 2;
+  const unsigned head_blocks = (unsigned)((kr + kHeadRows - 1) / kHeadRows);
+#define NGC_LAUNCH_HEAD(CP)                                                                                       \
+  do {                                                                                                            \
+    e = cudaFuncSetAttribute(mlp_head_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem);   \
+    if (e != cudaSuccess) return e;                                                                               \
+    mlp_head_kernel<CP><<<head_blocks, kHeadThreads, head_smem, stream>>>(H, hpad, hidden, C, W2, b2, y,          \
+                                                                          (long long)kr, D1, D2);                 \
+  } while (0)
+  if (cpad == 4) NGC_LAUNCH_HEAD(4);
+  else if (cpad == 8) NGC_LAUNCH_HEAD(8);
+  else if (cpad == 12) NGC_LAUNCH_HEAD(12);
+  else NGC_LAUNCH_HEAD(16);
+#undef NGC_LAUNCH_HEAD
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
   TnParams t;
   t.batch = k; t.status = status; t.num_k = (rows + 63) / 64;
   // [dW1; db1] = [X 1]^T delta1

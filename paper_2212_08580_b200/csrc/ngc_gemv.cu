@@ -459,55 +459,50 @@ combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const 
 }  // namespace
 
 namespace {
-// Encode for long gradients (dense models): every warp owns 128 columns and walks all n workers, holding
-// the sliding window of W >= s+1 group sums in registers, so each partial gradient is read once from
-// memory and never staged in shared memory.  Slots of the window beyond s carry a zero coefficient.
+// Encode for long gradients (dense models, one scratch slot per group): every thread owns 2 columns
+// and walks all n workers, holding a ring of W partial gradients in registers exactly as loaded
+// (fp32): s+1 of them form the worker's window, the other W-s-1 slots are loads still in flight for
+// the workers to come, and nothing touches a slot before its turn.  The arithmetic is done in the
+// type of the coded gradients (fp32 products and sums for fp32 storage).  Each partial gradient is
+// read once and never staged in shared memory.
 template <typename CT, int W>
 __global__ void __launch_bounds__(256)
-encode_stream_kernel(const RowSplit split, const float *__restrict__ ws, long long ld_ws,
-                     const double *__restrict__ coef, int n, int s, long long d, CT *__restrict__ coded) {
-  const long long col = (((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * 32 + (threadIdx.x & 31)) * 4;
+encode_stream_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n, int s,
+                     long long d, CT *__restrict__ coded) {
+  const long long col = ((long long)blockIdx.x * 256 + threadIdx.x) * 2;
   if (col >= d) return;
-  auto load_row = [&](int g, double (&r)[4]) {
-    const int c0 = split_owner(split, (long long)g * split.rows_g);
-    const int c1 = split_owner(split, (long long)(g + 1) * split.rows_g - 1);
-    const float *src = ws + ((size_t)g * split.P) * ld_ws + col;
-    r[0] = r[1] = r[2] = r[3] = 0.0;
-    for (int pce = 0; pce <= c1 - c0; ++pce) {
-      const float4 v = __ldg(reinterpret_cast<const float4 *>(src + (size_t)pce * ld_ws));
-      r[0] += (double)v.x; r[1] += (double)v.y; r[2] += (double)v.z; r[3] += (double)v.w;
-    }
-  };
-  double win[W][4];
+  const float *src = ws + col;
+  float2 win[W];
 #pragma unroll
-  for (int t = 0; t < W; ++t) load_row(t % n, win[t]);
-  const bool vec = (d % 4 == 0);
+  for (int t = 0; t < W; ++t) win[t] = __ldg(reinterpret_cast<const float2 *>(src + (size_t)(t % n) * ld_ws));
+  const bool pair = (d % 2 == 0);
+  int next = W % n;  // group that the next freed slot receives
   for (int i0 = 0; i0 < n; i0 += W) {
 #pragma unroll
     for (int t = 0; t < W; ++t) {
       const int i = i0 + t;
       if (i < n) {
-        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+        CT acc0 = 0, acc1 = 0;
+        const double *ci = coef + (size_t)i * (s + 1);
 #pragma unroll
         for (int k = 0; k < W; ++k) {
-          const double c = (k <= s) ? __ldg(coef + (size_t)i * (s + 1) + k) : 0.0;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[e] = fma(c, win[(t + k) % W][e], acc[e]);
+          if (k <= s) {
+            const CT c = (CT)__ldg(ci + k);
+            acc0 = fma(c, (CT)win[(t + k) % W].x, acc0);
+            acc1 = fma(c, (CT)win[(t + k) % W].y, acc1);
+          }
         }
         CT *dst = coded + (size_t)i * d + col;
-        if (vec) {
-          if (sizeof(CT) == 8) {
-            reinterpret_cast<double2 *>(dst)[0] = make_double2(acc[0], acc[1]);
-            reinterpret_cast<double2 *>(dst)[1] = make_double2(acc[2], acc[3]);
-          } else {
-            *reinterpret_cast<float4 *>(dst) = make_float4((float)acc[0], (float)acc[1], (float)acc[2], (float)acc[3]);
-          }
+        if (pair) {
+          if (sizeof(CT) == 8) *reinterpret_cast<double2 *>(dst) = make_double2((double)acc0, (double)acc1);
+          else *reinterpret_cast<float2 *>(dst) = make_float2((float)acc0, (float)acc1);
         } else {
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            if (col + e < d) dst[e] = (CT)acc[e];
+          dst[0] = acc0;
+          if (col + 1 < d) dst[1] = acc1;
         }
-        load_row((i + W) % n, win[t]);  // group i is no longer needed; its slot takes group i + W
+        // group i is no longer needed; its slot takes group i + W
+        win[t] = __ldg(reinterpret_cast<const float2 *>(src + (size_t)next * ld_ws));
+        if (++next == n) next = 0;
       }
     }
   }
@@ -537,16 +532,17 @@ encode_simple_kernel(const RowSplit split, const float *__restrict__ ws, long lo
 template <typename CT>
 cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long ld_ws, const double *coef, int n, int s,
                               long long d, CT *coded, cudaStream_t stream) {
-  const unsigned blocks = (unsigned)((d + 1023) / 1024);
-  if (s + 1 <= 4) encode_stream_kernel<CT, 4><<<blocks, 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
-  else if (s + 1 <= 8) encode_stream_kernel<CT, 8><<<blocks, 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
-  else if (s + 1 <= 12) encode_stream_kernel<CT, 12><<<blocks, 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
+  const unsigned blocks = (unsigned)((d + 511) / 512);
+  // ring size = window (s+1) plus at least two slots of loads in flight; one scratch slot per group only
+  if (split.P == 1 && s + 1 <= 2) encode_stream_kernel<CT, 4><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
+  else if (split.P == 1 && s + 1 <= 6) encode_stream_kernel<CT, 8><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
+  else if (split.P == 1 && s + 1 <= 12) encode_stream_kernel<CT, 16><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
   else encode_simple_kernel<CT><<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
   return cudaGetLastError();
 }
 }  // namespace
 
-// Encode for the dense models: ws holds [group][slot][ld_ws] fp32 with ld_ws a multiple of 4 and >= d.
+// Encode for the dense models: ws holds [group][slot][ld_ws] fp32, every slot filled, ld_ws a multiple of 4 and >= d.
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
                                int s, long long d, void *coded, int coded_dtype, cudaStream_t stream) {
   if (ld_ws % 4 != 0 || ld_ws < d) return cudaErrorInvalidValue;
