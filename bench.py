@@ -95,7 +95,7 @@ def algorithmic_flops(w: ngc_inputs.Workload) -> int:
 
 # dram__bytes_read + dram__bytes_write of the dominant kernel per full-size launch, from the ncu captures
 # summarised under profiles/ (None = not captured for the kernel as it stands).
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000}
 FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
 
 
