@@ -529,6 +529,313 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ------------------------------------------------------------------------------------------------
+// CTA-pair versions.  Two CTAs of a cluster (two SMs) drive one 256-row MMA (cta_group::2): each loads
+// its own 128 rows of A and only HALF of the 256-wide B tile, so the operand bytes an SM pulls from L2
+// per tensor-pipe cycle drop from 48 KB / 512 cycles to 32 KB / 512 cycles.  The leader CTA (cluster
+// rank 0) issues the MMAs for both; each CTA keeps its 128 accumulator rows in its own tensor memory and
+// runs its own epilogue.  Barriers: `full` lives in the leader and collects the TMA bytes of both CTAs;
+// `empty` and `tfull` exist in both and are signalled by a multicast commit; `tempty` lives in the leader
+// and counts the epilogue threads of both CTAs.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * 16384;  // 128 x 64 of A + 128 x 64 of B
+constexpr int kSmemPair = kPairStages * kPairStageBytes + 1024 + 256;
+
+struct PairSmem {
+  unsigned char *tiles;
+  uint32_t full[kPairStages], empty[kPairStages], tfull[2], tempty[2];
+  uint32_t *tmem_slot;
+};
+
+__device__ __forceinline__ PairSmem carve_pair(unsigned char *raw) {
+  PairSmem s;
+  const uint32_t base = smem_u32(raw);
+  s.tiles = raw + ((1024u - (base & 1023u)) & 1023u);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(s.tiles + kPairStages * kPairStageBytes);
+  for (int i = 0; i < kPairStages; ++i) {
+    s.full[i] = smem_u32(&bars[i]);
+    s.empty[i] = smem_u32(&bars[kPairStages + i]);
+  }
+  s.tfull[0] = smem_u32(&bars[2 * kPairStages]);
+  s.tfull[1] = smem_u32(&bars[2 * kPairStages + 1]);
+  s.tempty[0] = smem_u32(&bars[2 * kPairStages + 2]);
+  s.tempty[1] = smem_u32(&bars[2 * kPairStages + 3]);
+  s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kPairStages + 4]);
+  return s;
+}
+
+__device__ __forceinline__ uint32_t pair_prologue(const PairSmem &s, int warp) {
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kPairStages; ++i) {
+      mbar_init(s.full[i], 1);
+      mbar_init(s.empty[i], 1);
+    }
+    mbar_init(s.tfull[0], 1);
+    mbar_init(s.tfull[1], 1);
+    mbar_init(s.tempty[0], 256);
+    mbar_init(s.tempty[1], 256);
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(s.tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
+  tc_fence_after();
+  return *s.tmem_slot;
+}
+
+__device__ __forceinline__ void pair_teardown(int warp, uint32_t tmem_base, bool failed, int *status) {
+  if (failed) atomicExch(status, 1);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA leaves while the other may still touch its shared or tensor memory
+  if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kTcThreads, 1)
+fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const PairSmem s = carve_pair(smem_raw);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const uint32_t tmem_base = pair_prologue(s, warp);
+  bool failed = false;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  // p.row_blocks counts 256-row blocks here; this CTA owns rows [rb*256 + rank*128, +128)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int st = 0;
+      uint32_t ph = 0;
+      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
+        const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
+          if (rank == 0) mbar_expect_tx(s.full[st], 2 * kPairStageBytes);
+          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
+          const uint32_t bar = map_to_rank(s.full[st], 0);
+          tma_load_3d_pair(a, &tmX, kc * 64, rb * 256 + (int)rank * 128, j, bar);
+          tma_load_2d_pair(a + 16384, &tmW, kc * 64, nt * 256 + (int)rank * 128, bar);
+          if (++st == kPairStages) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = instr_desc_bf16(256, 256, 0, 0);
+      int st = 0, buf = 0;
+      uint32_t ph = 0, aph = 0;
+      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
+        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
+          const uint64_t ad = smem_desc_sw128(a, 16, 1024), bd = smem_desc_sw128(a + 16384, 16, 1024);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            mma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kc | k4) != 0);
+          mma_commit_pair(s.empty[st], 3);
+          if (++st == kPairStages) { st = 0; ph ^= 1u; }
+        }
+        if (failed) break;
+        mma_commit_pair(s.tfull[buf], 3);
+        buf ^= 1;
+        if (buf == 0) aph ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int buf = 0;
+    uint32_t aph = 0;
+    for (int tile = pair_id; tile < p.num_tiles; tile += n_pairs) {
+      const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
+      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
+      tc_fence_after();
+      const int row = rb * 256 + (int)rank * 128 + q * 32 + lane;
+      const bool valid = row < p.rows;
+      const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
+      __nv_bfloat16 *dst = p.out + grow * p.out_ld + nt * 256;
+      float v[32];
+      if (EPI == 0) {
+        const int label = valid ? p.y[grow] : -1;
+        float mx = -INFINITY;
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
+        }
+        float sum = 0.f;
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sum += __expf(v[i] - mx);
+        }
+        const float inv = 1.f / sum;
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const int c = c0 + g8 * 8 + h * 2;
+              const float r0 = __expf(v[g8 * 8 + h * 2] - mx) * inv - (c == label ? 1.f : 0.f);
+              const float r1 = __expf(v[g8 * 8 + h * 2 + 1] - mx) * inv - (c + 1 == label ? 1.f : 0.f);
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
+              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+            }
+            if (valid) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      } else {
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+          tmem_ld32(taddr + c0, v);
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const __nv_bfloat162 b2 =
+                  __floats2bfloat162_rn(fmaxf(v[g8 * 8 + h * 2], 0.f), fmaxf(v[g8 * 8 + h * 2 + 1], 0.f));
+              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+            }
+            if (valid) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        if (valid && nt == 0 && p.ones_col >= 0)
+          *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_rank(s.tempty[buf], 0));
+      buf ^= 1;
+      if (buf == 0) aph ^= 1u;
+    }
+  }
+  pair_teardown(warp, tmem_base, failed, p.status);
+}
+
+// Backward contraction on a CTA pair: tile = (batch j, 256 rows of M, 256 columns of N); N must be 256.
+__global__ void __launch_bounds__(kTcThreads, 1)
+tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TnParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const PairSmem s = carve_pair(smem_raw);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const uint32_t tmem_base = pair_prologue(s, warp);
+  bool failed = false;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int st = 0;
+      uint32_t ph = 0;
+      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
+        const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = tile / (p.n_tiles * p.m_tiles);
+        const int m0 = mt * 256 + (int)rank * 128, n0 = nt * 256 + (int)rank * 128;
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
+          if (rank == 0) mbar_expect_tx(s.full[st], 2 * kPairStageBytes);
+          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
+          const uint32_t bar = map_to_rank(s.full[st], 0);
+          tma_load_3d_pair(a, &tmA, m0, kc * 64, j, bar);
+          tma_load_3d_pair(a + 8192, &tmA, m0 + 64, kc * 64, j, bar);
+          tma_load_3d_pair(a + 16384, &tmB, n0, kc * 64, j, bar);
+          tma_load_3d_pair(a + 24576, &tmB, n0 + 64, kc * 64, j, bar);
+          if (++st == kPairStages) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = instr_desc_bf16(256, 256, 1, 1);
+      int st = 0, buf = 0;
+      uint32_t ph = 0, aph = 0;
+      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
+        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
+          const uint64_t ad = smem_desc_sw128(a, 8192, 1024), bd = smem_desc_sw128(a + 16384, 8192, 1024);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            mma_bf16_pair(acc, ad + (uint64_t)(k4 * 128), bd + (uint64_t)(k4 * 128), idesc, (kc | k4) != 0);
+          mma_commit_pair(s.empty[st], 3);
+          if (++st == kPairStages) { st = 0; ph ^= 1u; }
+        }
+        if (failed) break;
+        mma_commit_pair(s.tfull[buf], 3);
+        buf ^= 1;
+        if (buf == 0) aph ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int buf = 0;
+    uint32_t aph = 0;
+    const bool vec = (p.out_ld % 4 == 0) && (p.out_batch % 4 == 0);
+    for (int tile = pair_id; tile < p.num_tiles; tile += n_pairs) {
+      const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = tile / (p.n_tiles * p.m_tiles);
+      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
+      tc_fence_after();
+      const int m = mt * 256 + (int)rank * 128 + q * 32 + lane;
+      const bool valid = m < p.m_store;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
+      float *dst = p.out + (size_t)j * p.out_batch + (size_t)(valid ? m : 0) * p.out_ld + (size_t)nt * 256;
+      float v[32];
+      for (int c0 = 0; c0 < 256; c0 += 32) {
+        tmem_ld32(taddr + c0, v);
+        if (valid) {
+          if (vec) {
+#pragma unroll
+            for (int g4 = 0; g4 < 8; ++g4)
+              *reinterpret_cast<float4 *>(dst + c0 + g4 * 4) = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) dst[c0 + i] = v[i];
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_rank(s.tempty[buf], 0));
+      buf ^= 1;
+      if (buf == 0) aph ^= 1u;
+    }
+  }
+  pair_teardown(warp, tmem_base, failed, p.status);
+}
+
+// Launch on clusters of two CTAs.
+template <typename Kern, typename Params>
+cudaError_t launch_pair(Kern kern, int pair_tiles, int sms, const CUtensorMap &m0, const CUtensorMap &m1, const Params &p,
+                        cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPair);
+  if (e != cudaSuccess) return e;
+  int pairs = sms / 2;
+  if (pair_tiles < pairs) pairs = pair_tiles;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = kSmemPair;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, m0, m1, p);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Host side: tensor maps
 // ------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -607,21 +914,38 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
 
+  const bool pair = (C == 256) && sms >= 2;
   FwdParams p;
-  p.rows = rows; p.n_total = C; p.row_blocks = (rows + 127) / 128; p.n_tiles = 1;
-  p.num_tiles = k * p.row_blocks; p.num_k = (d + 63) / 64;
+  p.rows = rows; p.n_total = C; p.n_tiles = 1;
+  p.num_k = (d + 63) / 64;
   p.y = y; p.out = R; p.out_ld = C; p.ones_col = -1; p.status = status;
-  fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
-  e = cudaGetLastError();
+  if (pair) {
+    CUtensorMap tmWh;  // half of the class rows per CTA
+    const uint32_t wbox_h[2] = {64, 128};
+    if (!make_map(&tmWh, Wt, 2, wdims, wbox_h)) return cudaErrorInvalidValue;
+    p.row_blocks = (rows + 255) / 256;
+    p.num_tiles = k * p.row_blocks;
+    e = launch_pair(fwd_pair_kernel<0>, p.num_tiles, sms, tmXa, tmWh, p, stream);
+  } else {
+    p.row_blocks = (rows + 127) / 128;
+    p.num_tiles = k * p.row_blocks;
+    fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
+    e = cudaGetLastError();
+  }
   if (e != cudaSuccess) return e;
 
   TnParams t;
-  t.batch = k; t.m_tiles = (d + 127) / 128; t.n_tiles = 1; t.num_tiles = k * t.m_tiles;
+  t.batch = k; t.n_tiles = 1;
   t.num_k = (rows + 63) / 64;
   t.N = C; t.nbox = (C + 63) / 64;
   t.m_store = d; t.n_store = C;
   t.out = G; t.out_batch = (size_t)d * C; t.out_ld = C;
   t.status = status;
+  if (pair) {
+    t.m_tiles = (d + 255) / 256; t.num_tiles = k * t.m_tiles;
+    return launch_pair(tn_gemm_pair_kernel, t.num_tiles, sms, tmXb, tmR, t, stream);
+  }
+  t.m_tiles = (d + 127) / 128; t.num_tiles = k * t.m_tiles;
   tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmR, t);
   return cudaGetLastError();
 }
