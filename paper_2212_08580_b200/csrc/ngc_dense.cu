@@ -20,13 +20,19 @@ namespace {
 
 using namespace tc;
 
-constexpr int kStages = 4;
+constexpr int kStages = 4;     // backward kernel ring
+constexpr int kFwdStages = 3;  // forward kernel ring (the rest of shared memory stages the output tile)
 constexpr int kABytes = 128 * 64 * 2;  // 16 KB: 128 x 64 bf16
 constexpr int kBBytes = 256 * 64 * 2;  // 32 KB: 256 x 64 bf16
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 192;   // backward kernels: producer, MMA, 4 epilogue warps
+constexpr int kFwdThreads = 320;  // forward kernels: producer, MMA, 8 epilogue warps (two per tensor-memory quadrant)
+constexpr int kXchBytes = 2 * 2 * 128 * 4;  // row max / row sum exchanged between the two warps of a quadrant
 constexpr int kTmemCols = 512;
-constexpr int kSmemTc = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kStageLd = 264;  // bf16 elements per row of the output staging tile (256 + 8: conflict-free 16-byte rows)
+constexpr int kStageTileBytes = 128 * kStageLd * 2;
+constexpr int kSmemTc = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */ + kXchBytes;
+constexpr int kSmemFwd = kFwdStages * kStageBytes + 1024 + 256 + kXchBytes + kStageTileBytes;
 
 // Forward contraction D[128 rows x N] = X_tile[128 x K] * B^T with a fused epilogue.
 // Tile = (partition j, block of 128 rows, block nt of 256 output columns).
@@ -62,13 +68,17 @@ struct Smem {
   uint32_t full[kStages], empty[kStages], tfull[2], tempty[2];
   uint32_t *tmem_slot;
   volatile int *abort_flag;
+  float *xch;
+  __nv_bfloat16 *stage;  // forward kernels: 128 x kStageLd output staging tile
+  int nst;               // ring depth in use
 };
 
-__device__ __forceinline__ Smem carve(unsigned char *raw) {
+__device__ __forceinline__ Smem carve(unsigned char *raw, int nst) {
   Smem s;
   const uint32_t base = smem_u32(raw);
   s.tiles = raw + ((1024u - (base & 1023u)) & 1023u);
-  uint64_t *bars = reinterpret_cast<uint64_t *>(s.tiles + kStages * kStageBytes);
+  s.nst = nst;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(s.tiles + nst * kStageBytes);
   for (int i = 0; i < kStages; ++i) {
     s.full[i] = smem_u32(&bars[i]);
     s.empty[i] = smem_u32(&bars[kStages + i]);
@@ -79,20 +89,22 @@ __device__ __forceinline__ Smem carve(unsigned char *raw) {
   s.tempty[1] = smem_u32(&bars[2 * kStages + 3]);
   s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kStages + 4]);
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
+  s.xch = reinterpret_cast<float *>(s.tiles + nst * kStageBytes + 256);
+  s.stage = reinterpret_cast<__nv_bfloat16 *>(s.tiles + nst * kStageBytes + 256 + kXchBytes);
   return s;
 }
 
 // Common prologue: barriers, tensor memory.  Returns the tensor-memory base address.
-__device__ __forceinline__ uint32_t prologue(const Smem &s, int warp) {
+__device__ __forceinline__ uint32_t prologue(const Smem &s, int warp, int epi_threads) {
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kStages; ++i) {
+    for (int i = 0; i < s.nst; ++i) {
       mbar_init(s.full[i], 1);
       mbar_init(s.empty[i], 1);
     }
     mbar_init(s.tfull[0], 1);
     mbar_init(s.tfull[1], 1);
-    mbar_init(s.tempty[0], 128);
-    mbar_init(s.tempty[1], 128);
+    mbar_init(s.tempty[0], epi_threads);
+    mbar_init(s.tempty[1], epi_threads);
     *s.abort_flag = 0;
     mbar_fence_init();
   }
@@ -170,17 +182,116 @@ __global__ void convert_x_kernel(const float *__restrict__ X, __nv_bfloat16 *__r
   *reinterpret_cast<uint4 *>(Xb + row * ld + c0) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// Epilogues of the forward contractions.  Two threads share an accumulator row (same tensor-memory lane,
+// warps w and w + 4): thread `half` owns the 32-column chunks [c_lo, c_lo + nch), at most 4 of them.  All of
+// them are pulled into registers with back-to-back tensor-memory loads and one wait, after which the
+// accumulator buffer is handed back to the MMA warp (`release()`), before any arithmetic.
+//
+// Softmax residual R = softmax(z) - onehot(label), rounded to bf16: row max and row sum are exchanged through
+// `xch` ([2][2][128] floats) and a 64-thread named barrier per lane quadrant; one exponential per element.
+template <typename Release>
+__device__ __forceinline__ void softmax_residual_row(uint32_t taddr, int ncol, int c_lo, int nch, int label,
+                                                     __nv_bfloat16 *srow, float *xch, int rt, int half, int bar_id,
+                                                     Release release) {
+  constexpr float kLog2e = 1.4426950408889634f;
+  uint32_t r[128];
+  tmem_ld_chunks<4>(taddr + c_lo * 32, nch, r);
+  release();
+  const int nmine = min(ncol - c_lo * 32, nch * 32);  // columns of this thread (multiple of 16, may be <= 0)
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 128; i += 4) {
+    if (i < nmine) {
+      m0 = fmaxf(m0, __uint_as_float(r[i]));
+      m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
+      m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
+      m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+    }
+  }
+  xch[half * 128 + rt] = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+  asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+  const float mxs = fmaxf(xch[rt], xch[128 + rt]) * kLog2e;
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 128; i += 4) {
+    const bool in = i < nmine;
+    const float e0 = in ? exp2f(fmaf(__uint_as_float(r[i]), kLog2e, -mxs)) : 0.f;
+    const float e1 = in ? exp2f(fmaf(__uint_as_float(r[i + 1]), kLog2e, -mxs)) : 0.f;
+    const float e2 = in ? exp2f(fmaf(__uint_as_float(r[i + 2]), kLog2e, -mxs)) : 0.f;
+    const float e3 = in ? exp2f(fmaf(__uint_as_float(r[i + 3]), kLog2e, -mxs)) : 0.f;
+    s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+    r[i] = __float_as_uint(e0); r[i + 1] = __float_as_uint(e1);
+    r[i + 2] = __float_as_uint(e2); r[i + 3] = __float_as_uint(e3);
+  }
+  xch[256 + half * 128 + rt] = (s0 + s1) + (s2 + s3);
+  asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+  const float inv = 1.f / (xch[256 + rt] + xch[256 + 128 + rt]);
+  const int lm = label - c_lo * 32;  // position of the label among this thread's columns
+  asm volatile("bar.sync 5, 256;" ::: "memory");  // the previous tile has left the staging buffer
+#pragma unroll
+  for (int g8 = 0; g8 < 16; ++g8) {  // 8 values = one 16-byte store
+    uint32_t w[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const int i = g8 * 8 + h * 2;
+      const float r0 = __uint_as_float(r[i]) * inv - (i == lm ? 1.f : 0.f);
+      const float r1 = __uint_as_float(r[i + 1]) * inv - (i + 1 == lm ? 1.f : 0.f);
+      const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
+      w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+    }
+    if (g8 * 8 < nmine) *reinterpret_cast<uint4 *>(srow + c_lo * 32 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// H = relu(z), rounded to bf16.
+template <typename Release>
+__device__ __forceinline__ void relu_row(uint32_t taddr, int ncol, int c_lo, int nch, __nv_bfloat16 *srow,
+                                         Release release) {
+  uint32_t r[128];
+  tmem_ld_chunks<4>(taddr + c_lo * 32, nch, r);
+  release();
+  const int nmine = min(ncol - c_lo * 32, nch * 32);
+  asm volatile("bar.sync 5, 256;" ::: "memory");  // the previous tile has left the staging buffer
+#pragma unroll
+  for (int g8 = 0; g8 < 16; ++g8) {
+    uint32_t w[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const int i = g8 * 8 + h * 2;
+      const __nv_bfloat162 b2 =
+          __floats2bfloat162_rn(fmaxf(__uint_as_float(r[i]), 0.f), fmaxf(__uint_as_float(r[i + 1]), 0.f));
+      w[h] = *reinterpret_cast<const uint32_t *>(&b2);
+    }
+    if (g8 * 8 < nmine) *reinterpret_cast<uint4 *>(srow + c_lo * 32 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// Copies the staged 128 x ncol bf16 tile to global memory with full-row (coalesced) warp stores: each of the
+// 8 epilogue warps takes 16 rows.  `out_row0` points at column 0 of the tile's first row; rows beyond
+// `nrows` do not exist.
+__device__ __forceinline__ void store_staged_tile(const __nv_bfloat16 *stage, __nv_bfloat16 *out_row0, int out_ld,
+                                                  int nrows, int ncol, int epi_warp, int lane) {
+  if (lane * 8 < ncol) {
+#pragma unroll 4
+    for (int rr = epi_warp * 16; rr < epi_warp * 16 + 16; ++rr) {
+      if (rr < nrows)
+        *reinterpret_cast<uint4 *>(out_row0 + (size_t)rr * out_ld + lane * 8) =
+            *reinterpret_cast<const uint4 *>(stage + rr * kStageLd + lane * 8);
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Forward contractions.  EPI = 0: softmax residual  R = softmax(Z) - onehot(y)  (needs all classes in one
 // tile).  EPI = 1: H = relu(Z) (first MLP layer; bias already folded into the contraction).
 // ------------------------------------------------------------------------------------------------
 template <int EPI>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ unsigned char smem_raw[];
-  const Smem s = carve(smem_raw);
+  const Smem s = carve(smem_raw, kFwdStages);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tmem_base = prologue(s, warp);
+  const uint32_t tmem_base = prologue(s, warp, kFwdThreads - 64);
   bool failed = false;
 
   if (warp == 0) {
@@ -195,7 +306,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
           tma_load_3d(a, &tmX, kc * 64, rb * 128, j, s.full[st]);
           tma_load_2d(a + kABytes, &tmW, kc * 64, nt * 256, s.full[st]);
-          if (++st == kStages) { st = 0; ph ^= 1u; }
+          if (++st == kFwdStages) { st = 0; ph ^= 1u; }
         }
       }
     }
@@ -218,7 +329,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
           for (int k4 = 0; k4 < 4; ++k4)  // 16 bf16 = 32 bytes along K per instruction
             mma_bf16(acc, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc, (kc | k4) != 0);
           mma_commit(s.empty[st]);
-          if (++st == kStages) { st = 0; ph ^= 1u; }
+          if (++st == kFwdStages) { st = 0; ph ^= 1u; }
         }
         if (failed) break;
         mma_commit(s.tfull[buf]);
@@ -227,73 +338,37 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
       }
     }
   } else {
-    const int q = warp & 3;  // the 32-lane quadrant of tensor memory this warp may read
+    const int q = warp & 3;            // the 32-lane quadrant of tensor memory this warp may read
+    const int half = (warp - 2) >> 2;  // warps w and w + 4 share a quadrant and split the columns
     int buf = 0;
     uint32_t aph = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
       if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
       tc_fence_after();
-      const int row = rb * 128 + q * 32 + lane;
+      const int rt = q * 32 + lane, row = rb * 128 + rt;
       const bool valid = row < p.rows;
       const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
       const int ncol = min(256, p.n_total - nt * 256);
-      __nv_bfloat16 *dst = p.out + grow * p.out_ld + nt * 256;
-      float v[32];
+      const int nchunks = (ncol + 31) >> 5, hc = (nchunks + 1) >> 1;
+      const int c_lo = half ? hc : 0, nch = half ? nchunks - hc : hc;  // this thread's 32-column chunks
+      __nv_bfloat16 *srow = s.stage + rt * kStageLd;
+      const uint32_t tempty_bar = s.tempty[buf];
+      auto release = [&]() {  // the accumulator values are in registers: the MMA warp may overwrite the buffer
+        tc_fence_before();
+        mbar_arrive(tempty_bar);
+      };
       if (EPI == 0) {
-        const int label = valid ? p.y[grow] : -1;
-        float mx = -INFINITY;
-        for (int c0 = 0; c0 < ncol; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c0 + i < ncol) mx = fmaxf(mx, v[i]);
-        }
-        float sum = 0.f;
-        for (int c0 = 0; c0 < ncol; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c0 + i < ncol) sum += __expf(v[i] - mx);
-        }
-        const float inv = 1.f / sum;
-        for (int c0 = 0; c0 < ncol; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            uint32_t w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const int c = c0 + g8 * 8 + h * 2;
-              const float r0 = __expf(v[g8 * 8 + h * 2] - mx) * inv - (c == label ? 1.f : 0.f);
-              const float r1 = __expf(v[g8 * 8 + h * 2 + 1] - mx) * inv - (c + 1 == label ? 1.f : 0.f);
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
-              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
-            }
-            if (valid && c0 + g8 * 8 < ncol) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
+        softmax_residual_row(taddr, ncol, c_lo, nch, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release);
       } else {
-        for (int c0 = 0; c0 < ncol; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            uint32_t w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const __nv_bfloat162 b2 =
-                  __floats2bfloat162_rn(fmaxf(v[g8 * 8 + h * 2], 0.f), fmaxf(v[g8 * 8 + h * 2 + 1], 0.f));
-              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
-            }
-            if (valid && c0 + g8 * 8 < ncol) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-        if (valid && nt == 0 && p.ones_col >= 0)  // bf16 1.0 followed by zeros
+        relu_row(taddr, ncol, c_lo, nch, srow, release);
+        if (valid && half == 0 && nt == 0 && p.ones_col >= 0)  // bf16 1.0 followed by zeros
           *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
       }
-      tc_fence_before();
-      mbar_arrive(s.tempty[buf]);
+      asm volatile("bar.sync 5, 256;" ::: "memory");  // the tile is complete in shared memory
+      store_staged_tile(s.stage, p.out + ((size_t)j * p.rows + rb * 128) * p.out_ld + nt * 256, p.out_ld,
+                        p.rows - rb * 128, ncol, warp - 2, lane);
       buf ^= 1;
       if (buf == 0) aph ^= 1u;
     }
@@ -439,9 +514,9 @@ mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C
 __global__ void __launch_bounds__(kTcThreads, 1)
 tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TnParams p) {
   extern __shared__ unsigned char smem_raw[];
-  const Smem s = carve(smem_raw);
+  const Smem s = carve(smem_raw, kStages);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tmem_base = prologue(s, warp);
+  const uint32_t tmem_base = prologue(s, warp, kTcThreads - 64);
   bool failed = false;
 
   if (warp == 0) {
@@ -537,14 +612,16 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // `empty` and `tfull` exist in both and are signalled by a multicast commit; `tempty` lives in the leader
 // and counts the epilogue threads of both CTAs.
 // ------------------------------------------------------------------------------------------------
-constexpr int kPairStages = 6;
+constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = 2 * 16384;  // 128 x 64 of A + 128 x 64 of B
-constexpr int kSmemPair = kPairStages * kPairStageBytes + 1024 + 256;
+constexpr int kSmemPair = kPairStages * kPairStageBytes + 1024 + 256 + kXchBytes + kStageTileBytes;
 
 struct PairSmem {
   unsigned char *tiles;
   uint32_t full[kPairStages], empty[kPairStages], tfull[2], tempty[2];
   uint32_t *tmem_slot;
+  float *xch;
+  __nv_bfloat16 *stage;
 };
 
 __device__ __forceinline__ PairSmem carve_pair(unsigned char *raw) {
@@ -561,10 +638,12 @@ __device__ __forceinline__ PairSmem carve_pair(unsigned char *raw) {
   s.tempty[0] = smem_u32(&bars[2 * kPairStages + 2]);
   s.tempty[1] = smem_u32(&bars[2 * kPairStages + 3]);
   s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kPairStages + 4]);
+  s.xch = reinterpret_cast<float *>(s.tiles + kPairStages * kPairStageBytes + 256);
+  s.stage = reinterpret_cast<__nv_bfloat16 *>(s.tiles + kPairStages * kPairStageBytes + 256 + kXchBytes);
   return s;
 }
 
-__device__ __forceinline__ uint32_t pair_prologue(const PairSmem &s, int warp) {
+__device__ __forceinline__ uint32_t pair_prologue(const PairSmem &s, int warp, int epi_threads) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < kPairStages; ++i) {
       mbar_init(s.full[i], 1);
@@ -572,8 +651,8 @@ __device__ __forceinline__ uint32_t pair_prologue(const PairSmem &s, int warp) {
     }
     mbar_init(s.tfull[0], 1);
     mbar_init(s.tfull[1], 1);
-    mbar_init(s.tempty[0], 256);
-    mbar_init(s.tempty[1], 256);
+    mbar_init(s.tempty[0], 2 * epi_threads);
+    mbar_init(s.tempty[1], 2 * epi_threads);
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(s.tmem_slot), kTmemCols);
@@ -593,13 +672,13 @@ __device__ __forceinline__ void pair_teardown(int warp, uint32_t tmem_base, bool
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ unsigned char smem_raw[];
   const PairSmem s = carve_pair(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
-  const uint32_t tmem_base = pair_prologue(s, warp);
+  const uint32_t tmem_base = pair_prologue(s, warp, kFwdThreads - 64);
   bool failed = false;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   // p.row_blocks counts 256-row blocks here; this CTA owns rows [rb*256 + rank*128, +128)
@@ -649,69 +728,34 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     }
   } else {
     const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
     int buf = 0;
     uint32_t aph = 0;
     for (int tile = pair_id; tile < p.num_tiles; tile += n_pairs) {
       const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
       if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
       tc_fence_after();
-      const int row = rb * 256 + (int)rank * 128 + q * 32 + lane;
+      const int rt = q * 32 + lane, row = rb * 256 + (int)rank * 128 + rt;
       const bool valid = row < p.rows;
       const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
-      __nv_bfloat16 *dst = p.out + grow * p.out_ld + nt * 256;
-      float v[32];
+      const int c_lo = half ? 4 : 0;  // this thread's four 32-column chunks of the 256
+      __nv_bfloat16 *srow = s.stage + rt * kStageLd;
+      const uint32_t tempty_bar = map_to_rank(s.tempty[buf], 0);
+      auto release = [&]() {
+        tc_fence_before();
+        mbar_arrive_cluster(tempty_bar);
+      };
       if (EPI == 0) {
-        const int label = valid ? p.y[grow] : -1;
-        float mx = -INFINITY;
-        for (int c0 = 0; c0 < 256; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
-        }
-        float sum = 0.f;
-        for (int c0 = 0; c0 < 256; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) sum += __expf(v[i] - mx);
-        }
-        const float inv = 1.f / sum;
-        for (int c0 = 0; c0 < 256; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            uint32_t w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const int c = c0 + g8 * 8 + h * 2;
-              const float r0 = __expf(v[g8 * 8 + h * 2] - mx) * inv - (c == label ? 1.f : 0.f);
-              const float r1 = __expf(v[g8 * 8 + h * 2 + 1] - mx) * inv - (c + 1 == label ? 1.f : 0.f);
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
-              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
-            }
-            if (valid) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
+        softmax_residual_row(taddr, 256, c_lo, 4, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release);
       } else {
-        for (int c0 = 0; c0 < 256; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            uint32_t w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const __nv_bfloat162 b2 =
-                  __floats2bfloat162_rn(fmaxf(v[g8 * 8 + h * 2], 0.f), fmaxf(v[g8 * 8 + h * 2 + 1], 0.f));
-              w[h] = *reinterpret_cast<const uint32_t *>(&b2);
-            }
-            if (valid) *reinterpret_cast<uint4 *>(dst + c0 + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-        if (valid && nt == 0 && p.ones_col >= 0)
+        relu_row(taddr, 256, c_lo, 4, srow, release);
+        if (valid && half == 0 && nt == 0 && p.ones_col >= 0)
           *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
       }
-      tc_fence_before();
-      mbar_arrive_cluster(map_to_rank(s.tempty[buf], 0));
+      asm volatile("bar.sync 5, 256;" ::: "memory");
+      store_staged_tile(s.stage, p.out + ((size_t)j * p.rows + rb * 256 + (int)rank * 128) * p.out_ld + nt * 256,
+                        p.out_ld, p.rows - rb * 256 - (int)rank * 128, 256, warp - 2, lane);
       buf ^= 1;
       if (buf == 0) aph ^= 1u;
     }
@@ -726,7 +770,7 @@ tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const PairSmem s = carve_pair(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
-  const uint32_t tmem_base = pair_prologue(s, warp);
+  const uint32_t tmem_base = pair_prologue(s, warp, kTcThreads - 64);
   bool failed = false;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
@@ -814,15 +858,15 @@ tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 // Launch on clusters of two CTAs.
 template <typename Kern, typename Params>
-cudaError_t launch_pair(Kern kern, int pair_tiles, int sms, const CUtensorMap &m0, const CUtensorMap &m1, const Params &p,
-                        cudaStream_t stream) {
+cudaError_t launch_pair(Kern kern, int threads, int pair_tiles, int sms, const CUtensorMap &m0, const CUtensorMap &m1,
+                        const Params &p, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPair);
   if (e != cudaSuccess) return e;
   int pairs = sms / 2;
   if (pair_tiles < pairs) pairs = pair_tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
-  cfg.blockDim = dim3(kTcThreads);
+  cfg.blockDim = dim3(threads);
   cfg.dynamicSmemBytes = kSmemPair;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -909,7 +953,7 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
-  e = cudaFuncSetAttribute(fwd_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
+  e = cudaFuncSetAttribute(fwd_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFwd);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
@@ -925,11 +969,11 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
     if (!make_map(&tmWh, Wt, 2, wdims, wbox_h)) return cudaErrorInvalidValue;
     p.row_blocks = (rows + 255) / 256;
     p.num_tiles = k * p.row_blocks;
-    e = launch_pair(fwd_pair_kernel<0>, p.num_tiles, sms, tmXa, tmWh, p, stream);
+    e = launch_pair(fwd_pair_kernel<0>, kFwdThreads, p.num_tiles, sms, tmXa, tmWh, p, stream);
   } else {
     p.row_blocks = (rows + 127) / 128;
     p.num_tiles = k * p.row_blocks;
-    fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
+    fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream>>>(tmXa, tmW, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
@@ -943,7 +987,7 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   t.status = status;
   if (pair) {
     t.m_tiles = (d + 255) / 256; t.num_tiles = k * t.m_tiles;
-    return launch_pair(tn_gemm_pair_kernel, t.num_tiles, sms, tmXb, tmR, t, stream);
+    return launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, tmXb, tmR, t, stream);
   }
   t.m_tiles = (d + 127) / 128; t.num_tiles = k * t.m_tiles;
   tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmR, t);
@@ -1003,7 +1047,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   transpose_to_bf16_kernel<<<tg, tb, 0, stream>>>(W1, b1, W1t, d, hidden, dpad);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-  e = cudaFuncSetAttribute(fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
+  e = cudaFuncSetAttribute(fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFwd);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
@@ -1013,8 +1057,19 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   p.rows = rows; p.n_total = hidden; p.row_blocks = (rows + 127) / 128; p.n_tiles = (hidden + 255) / 256;
   p.num_tiles = k * p.row_blocks * p.n_tiles; p.num_k = (dpad + 63) / 64;
   p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = hidden; p.status = status;
-  fwd_kernel<1><<<p.num_tiles < sms ? p.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXa, tmW, p);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  const bool pair = (hidden % 256 == 0) && sms >= 2;  // CTA pairs: 256 rows per tile, half of W1^T per CTA
+  if (pair) {
+    CUtensorMap tmWh;
+    const uint32_t wbox_h[2] = {64, 128};
+    if (!make_map(&tmWh, W1t, 2, wdims, wbox_h)) return cudaErrorInvalidValue;
+    p.row_blocks = (rows + 255) / 256;
+    p.num_tiles = k * p.row_blocks * p.n_tiles;
+    e = launch_pair(fwd_pair_kernel<1>, kFwdThreads, p.num_tiles, sms, tmXa, tmWh, p, stream);
+  } else {
+    fwd_kernel<1><<<p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream>>>(tmXa, tmW, p);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) return e;
 
   const int cpad = (C + 3) / 4 * 4;
   const size_t head_smem = ((size_t)hidden * cpad + cpad + 4 * kHeadRows * cpad) * sizeof(float) + (size_t)kHeadRows * hpad * 2;
@@ -1040,8 +1095,14 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   t.N = hidden < 256 ? hidden : 256; t.nbox = (t.N + 63) / 64;
   t.m_store = d + 1; t.n_store = t.N;
   t.out = G; t.out_batch = lpad; t.out_ld = hidden;
-  tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmD1, t);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  if (pair) {
+    t.m_tiles = (d + 1 + 255) / 256; t.num_tiles = k * t.m_tiles * t.n_tiles;
+    e = launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, tmXb, tmD1, t, stream);
+  } else {
+    tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmD1, t);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) return e;
   // [dW2; db2] = [h 1]^T delta2
   t.m_tiles = (hidden + 1 + 127) / 128; t.n_tiles = 1; t.num_tiles = k * t.m_tiles;
   t.N = 16; t.nbox = 1;

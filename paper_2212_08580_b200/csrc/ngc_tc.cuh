@@ -112,6 +112,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 128 consecutive fp32 columns of this thread's lane: four loads issued back to back, one wait.  A
+// tensor-memory load has a long latency; issuing them one by one with a wait in between serialises it.
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+template <int NCHUNK>  // NCHUNK x 32 columns
+__device__ __forceinline__ void tmem_ld_chunks(uint32_t taddr, int nvalid, uint32_t (&r)[NCHUNK * 32]) {
+#pragma unroll
+  for (int c = 0; c < NCHUNK; ++c) {
+    if (c < nvalid) tmem_ld32_nowait(taddr + c * 32, &r[c * 32]);
+    else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) r[c * 32 + i] = 0u;
+    }
+  }
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  // every use of the registers has to come after the wait: route them through it
+#pragma unroll
+  for (int i = 0; i < NCHUNK * 32; ++i) asm volatile("" : "+r"(r[i]));
+}
+
 // ---- CTA pairs (cluster of two CTAs driving one 256-row MMA) ------------------------------------
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
