@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include "ngc_device.h"
+#include "ngc_f32x2.cuh"
 
 namespace ngc {
 
@@ -71,21 +72,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
-}
-
-// Two fp32 values in one 64-bit register pair, the operand type of the packed FMA.
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
-  f32x2 r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-// d = a * b + d on both halves (one issue slot for two fused multiply-adds).
-__device__ __forceinline__ void fma2(f32x2 &d, f32x2 a, f32x2 b) {
-  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
