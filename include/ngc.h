@@ -181,6 +181,13 @@ int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta
                   const void *y_host, const double *task_times_host, float *grad_host, ngc_step_info_t *info);
 
 /*
+ * Gradient-descent update of Eq. 1: theta <- theta - step * g with step = eta_t / m (the 1/m of Eq. 1 is
+ * the caller's: the decoded gradient is a plain sum).  theta_dev and grad_dev hold l floats; asynchronous
+ * on the stream, so it can be enqueued right behind ngc_step.
+ */
+int ngc_gd_update(float *theta_dev, const float *grad_dev, int64_t l, float step, void *cuda_stream);
+
+/*
  * Response-time model of Section II-D (Eq. 2 without the constants): task_times_host
  * [n][tasks] = shift + Exp(rate) i.i.d. from the SplitMix64 stream of `seed`; each
  * worker fails (all entries +inf) independently with probability p_fail.  Host only.
@@ -216,6 +223,25 @@ int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate,
 int ngc_grad_encode_static(const ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev,
                            const void *X_dev, const void *y_dev, int layer, void *coded_dev,
                            int32_t *status_dev, void *cuda_stream);
+
+/*
+ * Latency analysis of Section IV.
+ * ngc_latency_cdf_gc: Lemma 2, P(T_GC <= t) of an (n, k, sigma) gradient code.
+ * ngc_latency_cdf_ngc: Theorem 1, P(T_NGC <= t) of the fully nested (n, k, s_max) code (components 0..s_max).
+ * Per-task time = rho + Exp(lambda); gamma / eps the constant delays; workers fail independently with p_fail.
+ * Host only.  They return a negative number on invalid arguments.
+ * ngc_latency_mc: the same quantity by simulation for ANY plan: `trials` straggler patterns are drawn on the
+ * device (trial r uses the ngc_sample_times stream of seed SplitMix64(seed ^ 0xD1B54A32D192ED03, r + 1)), run
+ * through the stopping rule, and the latency (plan's gamma + eps + decode instant; +inf when no component ever
+ * becomes decodable) and the chosen level (-1 when none) are written to latency_dev[trials] / level_dev[trials]
+ * (device memory, either may be NULL).  Asynchronous on the stream.
+ */
+double ngc_latency_cdf_gc(int n, int sigma, double t, double lambda, double rho, double gamma, double eps,
+                          double p_fail);
+double ngc_latency_cdf_ngc(int n, int s_max, double t, double lambda, double rho, double gamma, double eps,
+                           double p_fail);
+int ngc_latency_mc(ngc_plan_t *plan, uint64_t seed, int64_t trials, double rho, double lambda, double p_fail,
+                   double *latency_dev, int32_t *level_dev, void *cuda_stream);
 
 /*
  * Timing of the dominant kernel of ngc_grad_encode (the fused gradient kernel).  While enabled,

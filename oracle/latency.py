@@ -6,7 +6,9 @@ match Lemma 2 (one component code) and Theorem 1 (nested code).
 """
 from __future__ import annotations
 
-from math import comb, exp, factorial
+from math import comb, exp, factorial, inf, log
+
+from .ngc_oracle import splitmix64_at
 
 
 def cdf_tasks(u: int, t: float, lam: float, rho: float, gamma: float, eps: float) -> float:
@@ -69,3 +71,24 @@ def cdf_ngc(t, n, s_max, lam, rho, gamma, eps, p_fail) -> float:
         cond = 1.0 - not_decodable(s_max + 1, 0, alive)
         total += cond * comb(n, kappa) * p_fail ** kappa * (1.0 - p_fail) ** (n - kappa)
     return total
+
+
+def sample_times(seed: int, n: int, tasks: int, shift: float, rate: float, p_fail: float):
+    """Response-time model of Section II-D from the SplitMix64 stream: worker i is dead when the uniform at
+    position 1 + i (tasks+1) is below p_fail; its m-th task takes shift - log(u) / rate with u the uniform
+    (bits + 1/2) / 2^53 at position 2 + i (tasks+1) + m."""
+    out = []
+    for i in range(n):
+        base = i * (tasks + 1)
+        dead = (splitmix64_at(seed, 1 + base) >> 11) / 9007199254740992.0 < p_fail
+        row = []
+        for m in range(tasks):
+            u = ((splitmix64_at(seed, 2 + base + m) >> 11) + 0.5) / 9007199254740992.0
+            row.append(inf if dead else shift - log(u) / rate)
+        out.append(row)
+    return out
+
+
+def trial_seed(seed: int, trial: int) -> int:
+    """Seed of Monte-Carlo trial `trial` of a run seeded with `seed`."""
+    return splitmix64_at(seed ^ 0xD1B54A32D192ED03, trial + 1)

@@ -75,6 +75,10 @@ def load_library() -> C.CDLL:
         "ngc_decode": (i32, [vp, i32, P(C.c_int32), i32, vp, i32, i64, vp, vp]),
         "ngc_step": (i32, [vp, P(Model), vp, vp, vp, P(dbl), vp, vp, P(StepInfo), vp]),
         "ngc_step_host": (i32, [vp, P(Model), vp, vp, vp, P(dbl), vp, P(StepInfo)]),
+        "ngc_latency_cdf_gc": (dbl, [i32, i32, dbl, dbl, dbl, dbl, dbl, dbl]),
+        "ngc_latency_cdf_ngc": (dbl, [i32, i32, dbl, dbl, dbl, dbl, dbl, dbl]),
+        "ngc_latency_mc": (i32, [vp, u64, i64, dbl, dbl, dbl, vp, vp, vp]),
+        "ngc_gd_update": (i32, [vp, vp, i64, C.c_float, vp]),
         "ngc_sample_times": (i32, [u64, i32, i32, dbl, dbl, dbl, P(dbl)]),
         "ngc_profile_enable": (i32, [vp, i32]),
         "ngc_profile_read": (i32, [vp, P(dbl), P(i64)]),
@@ -113,6 +117,23 @@ def sample_times(seed: int, n: int, tasks: int, shift: float, rate: float, p_fai
     if rc != 0:
         raise NgcError(rc, "ngc_sample_times")
     return out
+
+
+def latency_cdf_gc(n, sigma, t, lam, rho, gamma, eps, p_fail) -> float:
+    """Lemma 2: P(T_GC <= t)."""
+    return float(load_library().ngc_latency_cdf_gc(n, sigma, t, lam, rho, gamma, eps, p_fail))
+
+
+def latency_cdf_ngc(n, s_max, t, lam, rho, gamma, eps, p_fail) -> float:
+    """Theorem 1: P(T_NGC <= t) of the fully nested code."""
+    return float(load_library().ngc_latency_cdf_ngc(n, s_max, t, lam, rho, gamma, eps, p_fail))
+
+
+def gd_update(theta, grad, step: float, stream: int = 0):
+    """theta <- theta - step * grad on the device (Eq. 1 with step = eta / m)."""
+    rc = load_library().ngc_gd_update(_addr(theta), _addr(grad), int(theta.numel()), float(step), stream)
+    if rc != 0:
+        raise NgcError(rc, "ngc_gd_update")
 
 
 class Plan:
@@ -232,6 +253,11 @@ class Plan:
         self._check(self._lib.ngc_step_host(self._h, C.byref(model), _addr(theta), _addr(X), _addr(y), _dptr(t),
                                             _addr(grad), C.byref(info)), "ngc_step_host")
         return info
+
+    def latency_mc(self, seed: int, rho: float, lam: float, p_fail: float, latency, level, stream: int = 0):
+        """Monte Carlo of the stopping rule: fills the device tensors latency (float64) and level (int32)."""
+        self._check(self._lib.ngc_latency_mc(self._h, seed, int(latency.numel()), rho, lam, p_fail, _addr(latency),
+                                             _addr(level), stream), "ngc_latency_mc")
 
     def device_status(self) -> float:
         res = C.c_double()

@@ -322,6 +322,22 @@ int ngc_step_host(ngc_plan_t *p, const ngc_model_t *m, const float *theta, const
   return NGC_OK;
 }
 
+int ngc_latency_mc(ngc_plan_t *p, uint64_t seed, int64_t trials, double rho, double lambda, double p_fail,
+                   double *latency_dev, int32_t *level_dev, void *cuda_stream) {
+  if (!p || trials < 1 || !(rho >= 0.0) || !(lambda > 0.0) || !(p_fail >= 0.0 && p_fail <= 1.0)) return NGC_ERR_INVALID;
+  if (!latency_dev || !level_dev) return NGC_ERR_INVALID;
+  NGC_CUDA(p, ngc::launch_latency_mc(*p, seed, trials, rho, lambda, p_fail, latency_dev, level_dev,
+                                     static_cast<cudaStream_t>(cuda_stream)));
+  p->launches += 1;
+  return NGC_OK;
+}
+
+int ngc_gd_update(float *theta, const float *grad, int64_t l, float step, void *cuda_stream) {
+  if (!theta || !grad || l < 1 || !(step == step)) return NGC_ERR_INVALID;
+  return ngc::launch_gd_update(theta, grad, l, step, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NGC_OK
+                                                                                                            : NGC_ERR_CUDA;
+}
+
 size_t ngc_workspace_bytes(const ngc_plan_t *p) {
   if (!p) return 0;
   return p->ws_bytes + p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes + p->st_grad_bytes;

@@ -167,7 +167,18 @@ cudaError_t run_decode(const void *coded, const double *a, int n, long long l, f
   return cudaGetLastError();
 }
 
+__global__ void __launch_bounds__(256) gd_update_kernel(float *__restrict__ theta, const float *__restrict__ grad,
+                                                        long long l, float step) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < l) theta[i] = fmaf(-step, grad[i], theta[i]);
+}
+
 }  // namespace
+
+cudaError_t launch_gd_update(float *theta, const float *grad, long long l, float step, cudaStream_t stream) {
+  gd_update_kernel<<<(unsigned)((l + 255) / 256), 256, 0, stream>>>(theta, grad, l, step);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *masks_dev, MaskArg one, int batch,
                                 double *a_dev, double *resid_dev, double *maxres_dev, cudaStream_t stream) {

@@ -63,6 +63,14 @@ size_t softmax_scratch_bytes(int k, int rows, int d, int C);
 cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, const int *y, const float *W,
                                 unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream);
 
+// Monte Carlo of the stopping rule (Section IV): latency (gamma + eps + decode instant, +inf if never) and
+// chosen level (-1 if none) of `trials` seeded straggler patterns, into device buffers.
+cudaError_t launch_latency_mc(const ngc_plan_s &plan, uint64_t seed, long long trials, double shift, double rate,
+                              double p_fail, double *latency_dev, int *level_dev, cudaStream_t stream);
+
+// theta <- theta - step * grad (Eq. 1).
+cudaError_t launch_gd_update(float *theta, const float *grad, long long l, float step, cudaStream_t stream);
+
 int device_sm_count();
 
 }  // namespace ngc

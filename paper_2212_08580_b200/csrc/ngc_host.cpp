@@ -329,6 +329,85 @@ int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate,
   return NGC_OK;
 }
 
+// ---- Section IV closed forms ----------------------------------------------------------------------
+namespace {
+// Binomial coefficients as doubles, Pascal's rule.
+struct Binom {
+  std::vector<double> c;
+  int n;
+  explicit Binom(int n_) : c((size_t)(n_ + 1) * (n_ + 1), 0.0), n(n_) {
+    for (int a = 0; a <= n; ++a) {
+      c[(size_t)a * (n + 1)] = 1.0;
+      for (int b = 1; b <= a; ++b)
+        c[(size_t)a * (n + 1) + b] = c[(size_t)(a - 1) * (n + 1) + b - 1] + (b <= a - 1 ? c[(size_t)(a - 1) * (n + 1) + b] : 0.0);
+    }
+  }
+  double operator()(int a, int b) const { return (b < 0 || b > a) ? 0.0 : c[(size_t)a * (n + 1) + b]; }
+};
+
+// Eq. 3 with the Erlang tail summed over k = 0..u-1: P(u tasks done by t).
+double tasks_cdf(int u, double t, double lam, double rho, double gamma, double eps) {
+  if (u == 0) return 1.0;
+  const double x = t - (gamma + eps + u * rho);
+  if (x <= 0.0) return 0.0;
+  double term = 1.0, tail = 1.0;
+  for (int k = 1; k < u; ++k) {
+    term *= lam * x / k;
+    tail += term;
+  }
+  return 1.0 - tail * std::exp(-lam * x);
+}
+bool latency_args_ok(int n, int s, double lam, double rho, double gamma, double eps, double pf) {
+  return n >= 1 && n <= NGC_MAX_N && s >= 0 && s < n && lam > 0.0 && rho >= 0.0 && gamma >= 0.0 && eps >= 0.0 &&
+         pf >= 0.0 && pf <= 1.0;
+}
+}  // namespace
+
+double ngc_latency_cdf_gc(int n, int sigma, double t, double lam, double rho, double gamma, double eps, double pf) {
+  if (!latency_args_ok(n, sigma, lam, rho, gamma, eps, pf)) return -1.0;
+  const Binom C(n);
+  const double F = tasks_cdf(sigma + 1, t, lam, rho, gamma, eps);
+  double total = 0.0;
+  for (int kappa = 0; kappa <= sigma; ++kappa) {
+    const int alive = n - kappa;
+    double cond = 0.0;
+    for (int tau = n - sigma; tau <= alive; ++tau) cond += C(alive, tau) * std::pow(F, tau) * std::pow(1.0 - F, alive - tau);
+    total += cond * C(n, kappa) * std::pow(pf, kappa) * std::pow(1.0 - pf, n - kappa);
+  }
+  return total;
+}
+
+double ngc_latency_cdf_ngc(int n, int s_max, double t, double lam, double rho, double gamma, double eps, double pf) {
+  if (!latency_args_ok(n, s_max, lam, rho, gamma, eps, pf)) return -1.0;
+  const Binom C(n);
+  const int top = s_max + 1;
+  std::vector<double> F(top + 2), q(top + 1);
+  for (int u = 0; u <= top + 1; ++u) F[u] = tasks_cdf(u, t, lam, rho, gamma, eps);
+  for (int u = 0; u < top; ++u) q[u] = F[u] - F[u + 1];  // exactly u tasks done
+  q[top] = F[top];                                        // s_max + 1 (or more) done
+  double total = 0.0;
+  for (int kappa = 0; kappa <= s_max; ++kappa) {
+    const int alive = n - kappa;
+    // w[c] = weight of the configurations in which c alive workers have finished at least u tasks and no
+    // component has been decodable so far (at most n - v workers with >= v tasks, for every v >= u)
+    std::vector<double> w(alive + 1, 0.0), w2(alive + 1);
+    for (int c = 0; c <= std::min(alive, n - top); ++c) w[c] = C(alive, c) * std::pow(q[top], c);
+    for (int u = top - 1; u >= 1; --u) {
+      std::fill(w2.begin(), w2.end(), 0.0);
+      const int cap = std::min(alive, n - u);
+      for (int c = 0; c <= alive; ++c) {
+        if (w[c] == 0.0) continue;
+        for (int i = 0; c + i <= cap; ++i) w2[c + i] += w[c] * C(alive - c, i) * std::pow(q[u], i);
+      }
+      w.swap(w2);
+    }
+    double not_decodable = 0.0;
+    for (int c = 0; c <= alive; ++c) not_decodable += w[c] * std::pow(q[0], alive - c);
+    total += (1.0 - not_decodable) * C(n, kappa) * std::pow(pf, kappa) * std::pow(1.0 - pf, n - kappa);
+  }
+  return total;
+}
+
 const char *ngc_strerror(int status) {
   switch (status) {
     case NGC_OK: return "ok";
