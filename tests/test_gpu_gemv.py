@@ -29,6 +29,8 @@ CASES = [
     ("lsq", "bf16", 8, [2], 64, 8192, 1),                # single component code (plain gradient code)
     ("lsq", "f32", 4, [1, 2], 50, 256, 3),               # k = 3 n: atomic task = 3 partitions
     ("logistic", "f32", 3, [1], 1, 4, 1),                # one row, one vector
+    ("lsq", "f32", 128, [1, 32], 3, 64, 1),              # the largest n and the largest tolerance the library takes
+    ("lsq", "bf16", 2, [0, 1], 5000, 16384, 1),          # many rows per CTA range, widest rows
 ]
 
 
