@@ -509,6 +509,221 @@ mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C
 }
 
 // ------------------------------------------------------------------------------------------------
+// MLP head on the tensor cores (hidden a multiple of 64, at most 512; at most 16 classes).  Per tile of
+// 128 samples, everything stays in shared / tensor memory:
+//   1. TMA brings the 128 x hidden tile of h (bf16, K-major, 128-byte swizzle);
+//   2. z[128 x 16] = h W2 (W2^T resident in shared memory as the B operand, N = 16);
+//   3. one thread per sample: z + b2 -> softmax -> delta2; delta2 goes to global memory (for dW2) and, as
+//      a bf16 row of a swizzled 128 x 64 tile, becomes the A operand of the next contraction;
+//   4. (delta2 W2^T)[128 x hidden] with K = 16: one MMA per 256 hidden units;
+//   5. the threads mask by h > 0 (read from the tile in its swizzled layout), overwrite h by delta1 in
+//      place, and TMA stores the tile to delta1[rows][hidden].
+// ------------------------------------------------------------------------------------------------
+constexpr int kHeadTcThreads = 192;
+
+struct HeadTcParams {
+  int hidden, C, num_tiles;
+  const float *b2;
+  const int *y;
+  long long rows_total;
+  __nv_bfloat16 *D2;  // [rows_total][64]
+  int *status;
+};
+
+__global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, __nv_bfloat16 *__restrict__ W2t,
+                               __nv_bfloat16 *__restrict__ W2k) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < 16 * hidden) {  // W2t[c][hc]
+    const int c = i / hidden, hc = i % hidden;
+    W2t[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
+  }
+  if (i < hidden * 64) {  // W2k[hc][c]
+    const int hc = i / 64, c = i % 64;
+    W2k[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
+  }
+}
+
+__global__ void __launch_bounds__(kHeadTcThreads, 1)
+mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW2t,
+                   const __grid_constant__ CUtensorMap tmW2k, const __grid_constant__ CUtensorMap tmD1,
+                   const HeadTcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char *sm = smem_raw + ((1024u - (base & 1023u)) & 1023u);
+  const int nchunk = p.hidden / 64, nhalf = (p.hidden + 255) / 256;
+  unsigned char *htile = sm;                                  // nchunk x [128 x 64] bf16
+  unsigned char *d2tile = htile + (size_t)nchunk * 16384;     // [128 x 64] bf16 (16 columns used)
+  unsigned char *w2k = d2tile + 16384;                        // nhalf x [256 x 64] bf16
+  unsigned char *w2t = w2k + (size_t)nhalf * 32768;           // nchunk x [16 x 64] bf16
+  uint64_t *bars = reinterpret_cast<uint64_t *>(w2t + (size_t)nchunk * 2048);
+  const uint32_t h_full = smem_u32(&bars[0]), h_empty = smem_u32(&bars[1]), z_full = smem_u32(&bars[2]),
+                 d2_full = smem_u32(&bars[3]), d_full = smem_u32(&bars[4]), d_empty = smem_u32(&bars[5]),
+                 w_full = smem_u32(&bars[6]);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[7]);
+  float *b2s = reinterpret_cast<float *>(&bars[8]);           // 16 floats
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(h_full, 1);
+    mbar_init(h_empty, 1);
+    mbar_init(z_full, 1);
+    mbar_init(d2_full, 128);
+    mbar_init(d_full, 1);
+    mbar_init(d_empty, 128);
+    mbar_init(w_full, 1);
+    mbar_fence_init();
+  }
+  if (threadIdx.x < 16) b2s[threadIdx.x] = (int)threadIdx.x < p.C ? p.b2[threadIdx.x] : 0.f;
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t z_acc = tmem_base, d_acc = tmem_base + 256u;
+  bool failed = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(w_full, (uint32_t)(nchunk * 2048 + nhalf * 32768));
+      for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(w2t + kc * 2048), &tmW2t, kc * 64, 0, w_full);
+      for (int hh = 0; hh < nhalf; ++hh) tma_load_2d(smem_u32(w2k + hh * 32768), &tmW2k, 0, hh * 256, w_full);
+      uint32_t ph = 0;
+      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+        if (!mbar_wait(h_empty, ph ^ 1u)) { failed = true; break; }
+        mbar_expect_tx(h_full, (uint32_t)nchunk * 16384u);
+        for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(htile + kc * 16384), &tmH, kc * 64, tile * 128, h_full);
+        ph ^= 1u;
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_z = instr_desc_bf16(128, 16, 0, 0);
+      uint32_t ph = 0, dph = 0;
+      if (!mbar_wait(w_full, 0)) failed = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
+        if (!mbar_wait(h_full, ph)) { failed = true; break; }
+        tc_fence_after();
+        for (int kc = 0; kc < nchunk; ++kc) {
+          const uint64_t ad = smem_desc_sw128(smem_u32(htile + kc * 16384), 16, 1024);
+          const uint64_t bd = smem_desc_sw128(smem_u32(w2t + kc * 2048), 16, 1024);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            mma_bf16(z_acc, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc_z, (kc | k4) != 0);
+        }
+        mma_commit(z_full);
+        if (!mbar_wait(d2_full, ph)) { failed = true; break; }
+        tc_fence_after();
+        const uint64_t ad = smem_desc_sw128(smem_u32(d2tile), 16, 1024);
+        for (int hh = 0; hh < nhalf; ++hh) {
+          if (!mbar_wait(d_empty, dph ^ 1u)) { failed = true; break; }
+          tc_fence_after();
+          const int nh = min(256, p.hidden - hh * 256);
+          const uint64_t bd = smem_desc_sw128(smem_u32(w2k + hh * 32768), 16, 1024);
+          mma_bf16(d_acc, ad, bd, instr_desc_bf16(128, nh, 0, 0), 0);  // K = 16: the 16 class columns
+          mma_commit(d_full);
+          dph ^= 1u;
+        }
+        ph ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3, r = q * 32 + lane;  // row of the tile = tensor-memory lane
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;  // row r inside a swizzled tile
+    const uint32_t rx = (uint32_t)(r & 7);
+    uint32_t ph = 0, dph = 0;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const long long row = (long long)tile * 128 + r;
+      const bool valid = row < p.rows_total;
+      if (!mbar_wait(z_full, ph)) { failed = true; break; }
+      tc_fence_after();
+      float v[32];
+      tmem_ld32(z_acc + lane_off, v);
+      const int label = valid ? p.y[row] : -1;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        v[c] += b2s[c];
+        if (c < p.C) mx = fmaxf(mx, v[c]);
+      }
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        v[c] = c < p.C ? __expf(v[c] - mx) : 0.f;
+        sum += v[c];
+      }
+      const float inv = 1.f / sum;
+      uint32_t w[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float lo = (2 * u < p.C) ? v[2 * u] * inv - (2 * u == label ? 1.f : 0.f) : 0.f;
+        const float hi = (2 * u + 1 < p.C) ? v[2 * u + 1] * inv - (2 * u + 1 == label ? 1.f : 0.f) : 0.f;
+        const __nv_bfloat162 b2v = __floats2bfloat162_rn(lo, hi);
+        w[u] = *reinterpret_cast<const uint32_t *>(&b2v);
+      }
+      if (valid) {
+        uint4 *d2 = reinterpret_cast<uint4 *>(p.D2 + row * 64);
+        d2[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        d2[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      }
+      *reinterpret_cast<uint4 *>(d2tile + row_off + ((0u ^ rx) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4 *>(d2tile + row_off + ((1u ^ rx) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+      fence_async_smem();
+      mbar_arrive(d2_full);
+      // the threads read h themselves below: observe the completion of its TMA copies directly
+      if (!mbar_wait(h_full, ph)) { failed = true; break; }
+      for (int hh = 0; hh < nhalf; ++hh) {
+        if (!mbar_wait(d_full, dph)) { failed = true; break; }
+        tc_fence_after();
+        const int nh = min(256, p.hidden - hh * 256);
+        for (int gulp = 0; gulp * 128 < nh; ++gulp) {
+          uint32_t rr[128];
+          const int nch = min(4, (nh - gulp * 128) / 32);
+          tmem_ld_chunks<4>(d_acc + lane_off + gulp * 128, nch, rr);
+          if ((gulp + 1) * 128 >= nh) {  // the accumulator has been read completely
+            tc_fence_before();
+            mbar_arrive(d_empty);
+          }
+#pragma unroll
+          for (int g = 0; g < 16; ++g) {
+            if (g * 8 < nch * 32) {
+              const int col = hh * 256 + gulp * 128 + g * 8;  // hidden unit of the first of 8 values
+              unsigned char *hp = htile + (size_t)(col >> 6) * 16384 + row_off + ((((uint32_t)(col & 63) >> 3) ^ rx) << 4);
+              const uint4 hv = *reinterpret_cast<const uint4 *>(hp);
+              const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+              uint32_t o[4];
+#pragma unroll
+              for (int t2 = 0; t2 < 4; ++t2) {
+                const float d0 = __uint_as_float(hw[t2] << 16) > 0.f ? __uint_as_float(rr[g * 8 + 2 * t2]) : 0.f;
+                const float d1 = __uint_as_float(hw[t2] & 0xffff0000u) > 0.f ? __uint_as_float(rr[g * 8 + 2 * t2 + 1]) : 0.f;
+                const __nv_bfloat162 db = __floats2bfloat162_rn(d0, d1);
+                o[t2] = *reinterpret_cast<const uint32_t *>(&db);
+              }
+              *reinterpret_cast<uint4 *>(hp) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          }
+        }
+        dph ^= 1u;
+      }
+      if (failed) break;
+      // delta1 now sits where h was: hand the tile to TMA, then give the buffer back to the producer
+      fence_async_smem();
+      asm volatile("bar.sync 6, 128;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        for (int kc = 0; kc < nchunk; ++kc) tma_store_2d(&tmD1, kc * 64, tile * 128, smem_u32(htile + kc * 16384));
+        tma_store_commit_and_wait_read();
+        mbar_arrive(h_empty);
+      }
+      ph ^= 1u;
+    }
+  }
+  if (failed) atomicExch(p.status, 1);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Backward contractions: D = A^T B with K = the partition's rows (see TnParams).
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -1003,7 +1218,7 @@ size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
   const size_t l = (size_t)d * hidden + hidden + (size_t)hidden * C + C, lpad = (l + 3) / 4 * 4;
   const size_t kr = (size_t)k * rows;
   return up256(kr * dpad * 2) + up256((size_t)hidden * dpad * 2) + up256(kr * hpad * 2) + up256(kr * hidden * 2) +
-         up256(kr * 64 * 2) + up256((size_t)k * lpad * 4);
+         up256(kr * 64 * 2) + up256((size_t)16 * hidden * 2) + up256((size_t)hidden * 64 * 2) + up256((size_t)k * lpad * 4);
 }
 
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
@@ -1021,6 +1236,8 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   __nv_bfloat16 *H = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256(kr * hpad * 2);
   __nv_bfloat16 *D1 = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256(kr * hidden * 2);
   __nv_bfloat16 *D2 = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256(kr * 64 * 2);
+  __nv_bfloat16 *W2t = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)16 * hidden * 2);
+  __nv_bfloat16 *W2k = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)hidden * 64 * 2);
   float *G = reinterpret_cast<float *>(ptr);
   *G_out = G;
   *G_ld = (long long)lpad;
@@ -1071,9 +1288,30 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   }
   if (e != cudaSuccess) return e;
 
-  const int cpad = (C + 3) / 4 * 4;
-  const size_t head_smem = ((size_t)hidden * cpad + cpad + 4 * kHeadRows * cpad) * sizeof(float) + (size_t)kHeadRows * hpad * 2;
-  const unsigned head_blocks = (unsigned)((kr + kHeadRows - 1) / kHeadRows);
+  const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
+  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 256 + 1024;
+  if (hidden % 64 == 0 && head_tc_smem <= 232448) {
+    CUtensorMap tmH2, tmW2t, tmW2k, tmD1s;
+    const uint64_t h2dims[2] = {(uint64_t)hpad, (uint64_t)kr}, w2tdims[2] = {(uint64_t)hidden, 16},
+                   w2kdims[2] = {64, (uint64_t)hidden}, d1sdims[2] = {(uint64_t)hidden, (uint64_t)kr};
+    const uint32_t box_h[2] = {64, 128}, box_w2t[2] = {64, 16}, box_w2k[2] = {64, 256};
+    if (!make_map(&tmH2, H, 2, h2dims, box_h) || !make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) ||
+        !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) || !make_map(&tmD1s, D1, 2, d1sdims, box_h))
+      return cudaErrorInvalidValue;
+    prep_w2_kernel<<<(hidden * 64 + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    HeadTcParams hp;
+    hp.hidden = hidden; hp.C = C; hp.num_tiles = (int)((kr + 127) / 128);
+    hp.b2 = b2; hp.y = y; hp.rows_total = (long long)kr; hp.D2 = D2; hp.status = status;
+    e = cudaFuncSetAttribute(mlp_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_tc_smem);
+    if (e != cudaSuccess) return e;
+    mlp_head_tc_kernel<<<hp.num_tiles < sms ? hp.num_tiles : sms, kHeadTcThreads, head_tc_smem, stream>>>(
+        tmH2, tmW2t, tmW2k, tmD1s, hp);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  } else {
+    const int cpad = (C + 3) / 4 * 4;
+    const size_t head_smem = ((size_t)hidden * cpad + cpad + 4 * kHeadRows * cpad) * sizeof(float) + (size_t)kHeadRows * hpad * 2;
+    const unsigned head_blocks = (unsigned)((kr + kHeadRows - 1) / kHeadRows);
 #define NGC_LAUNCH_HEAD(CP)                                                                                       \
   do {                                                                                                            \
     e = cudaFuncSetAttribute(mlp_head_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem);   \
@@ -1081,12 +1319,13 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     mlp_head_kernel<CP><<<head_blocks, kHeadThreads, head_smem, stream>>>(H, hpad, hidden, C, W2, b2, y,          \
                                                                           (long long)kr, D1, D2);                 \
   } while (0)
-  if (cpad == 4) NGC_LAUNCH_HEAD(4);
-  else if (cpad == 8) NGC_LAUNCH_HEAD(8);
-  else if (cpad == 12) NGC_LAUNCH_HEAD(12);
-  else NGC_LAUNCH_HEAD(16);
+    if (cpad == 4) NGC_LAUNCH_HEAD(4);
+    else if (cpad == 8) NGC_LAUNCH_HEAD(8);
+    else if (cpad == 12) NGC_LAUNCH_HEAD(12);
+    else NGC_LAUNCH_HEAD(16);
 #undef NGC_LAUNCH_HEAD
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
 
   TnParams t;
   t.batch = k; t.status = status; t.num_k = (rows + 63) / 64;

@@ -67,6 +67,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
       : "memory");
 }
 
+// TMA store of one box from shared memory (same swizzled layout as the loads); rows beyond the tensor are
+// clipped.  commit + wait_read: afterwards the shared-memory source may be overwritten.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int c0, int c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(c0),
+               "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit_and_wait_read() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// Makes this thread's ordinary shared-memory writes visible to TMA / tcgen05 (the async proxy).
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // ---- tensor memory ----------------------------------------------------------------------------
 // Whole-warp calls.  `cols` is a power of two in [32, 512].
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
