@@ -155,6 +155,9 @@ void ngc_plan_destroy(ngc_plan_t *p) {
     cudaFree(p->st_grad);
   }
   for (void *e : p->ev) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+  if (p->ev_solved) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_solved));
+  if (p->ev_decoded) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_decoded));
+  if (p->side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(p->side_stream));
   delete p;
 }
 
@@ -279,10 +282,15 @@ int ngc_decode(ngc_plan_t *p, int layer, const int32_t *S, int nS, const void *c
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
   NGC_CUDA(p, ngc::launch_decode(coded, coded_dtype, p->d_a, p->n, l, grad, stream));
+  if (p->ev_decoded) NGC_CUDA(p, cudaEventRecord(static_cast<cudaEvent_t>(p->ev_decoded), stream));
   p->launches += 2;
   return NGC_OK;
 }
 
+// The decoding vector depends only on the responsive set, which is known before any gradient is:
+// ngc_step solves it on a stream of the plan's own, under the gradient kernels, and the decode on the
+// caller's stream waits for it.  The solve of one step in turn waits until the decode of the step
+// before has read the vector.  A capturing stream takes the plain in-order path.
 int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y,
              const double *task_times, void *coded, float *grad, ngc_step_info_t *info, void *cuda_stream) {
   if (!p || !info) return NGC_ERR_INVALID;
@@ -290,10 +298,50 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
   if (rc != NGC_OK) return rc;
   rc = ngc_select(p, task_times, info);
   if (rc != NGC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  NGC_CUDA(p, cudaStreamIsCapturing(stream, &cap));
+  // A gradient CTA that fills its SM's register file would have to wait for the solve's block to leave
+  // (and the solve is slow under a bandwidth-bound kernel): such models keep the in-order path.
+  if (p->overlap_kind != m->kind || p->overlap_d != m->d || p->overlap_dtype != m->x_dtype) {
+    p->overlap_kind = m->kind; p->overlap_d = m->d; p->overlap_dtype = m->x_dtype;
+    p->overlap_ok = (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) ? ngc::gemv_pair_leaves_room(*m) : true;
+  }
+  if (!p->overlap_ok || cap != cudaStreamCaptureStatusNone || !coded || !grad || !aligned16(coded)) {
+    rc = ngc_grad_encode(p, m, theta, X, y, info->layer, coded, cuda_stream);
+    if (rc != NGC_OK) return rc;
+    return ngc_decode(p, info->layer, info->S, info->nS, coded, ngc_coded_dtype(p, m), ngc_num_params(m), grad,
+                      cuda_stream);
+  }
+  ngc::MaskArg mask;
+  rc = pack_set(p, info->layer, info->S, info->nS, mask.w);
+  if (rc != NGC_OK) return rc;
+  if ((rc = ensure_tables(p)) != NGC_OK) return rc;
+  if ((rc = ensure_batch(p, 1)) != NGC_OK) return rc;
+  if (!p->side_stream) {
+    cudaStream_t s2;
+    cudaEvent_t e1, e2;
+    NGC_CUDA(p, cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking));
+    p->side_stream = s2;
+    NGC_CUDA(p, cudaEventCreateWithFlags(&e1, cudaEventDisableTiming));
+    p->ev_solved = e1;
+    NGC_CUDA(p, cudaEventCreateWithFlags(&e2, cudaEventDisableTiming));
+    p->ev_decoded = e2;
+    // everything already queued on the caller's stream (an earlier ngc_decode, say) comes first
+    NGC_CUDA(p, cudaEventRecord(e2, stream));
+  }
+  cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);
+  cudaEvent_t solved = static_cast<cudaEvent_t>(p->ev_solved), decoded = static_cast<cudaEvent_t>(p->ev_decoded);
+  NGC_CUDA(p, cudaStreamWaitEvent(side, decoded, 0));
+  NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
+  NGC_CUDA(p, cudaEventRecord(solved, side));
   rc = ngc_grad_encode(p, m, theta, X, y, info->layer, coded, cuda_stream);
   if (rc != NGC_OK) return rc;
-  return ngc_decode(p, info->layer, info->S, info->nS, coded, ngc_coded_dtype(p, m), ngc_num_params(m), grad,
-                    cuda_stream);
+  NGC_CUDA(p, cudaStreamWaitEvent(stream, solved, 0));
+  NGC_CUDA(p, ngc::launch_decode(coded, ngc_coded_dtype(p, m), p->d_a, p->n, ngc_num_params(m), grad, stream));
+  NGC_CUDA(p, cudaEventRecord(decoded, stream));
+  p->launches += 2;
+  return NGC_OK;
 }
 
 int ngc_step_host(ngc_plan_t *p, const ngc_model_t *m, const float *theta, const void *X, const void *y,

@@ -17,19 +17,30 @@ namespace {
 // ------------------------------------------------------------------------------------------
 constexpr int kSolveWarps = 4;
 
+// Shared memory of one warp: M[s][s+1], z[s], a[n] doubles, then the list of unused workers and the
+// used flags.  Sized by the level, so that a single-pattern solve (one warp, about 2 KB) finds room
+// on an SM beside a resident gradient CTA and can run under it.
+__host__ __device__ inline size_t solve_warp_bytes(int n, int s) {
+  const size_t dbl = (size_t)s * (s + 1) + s + n;
+  const size_t tail = (size_t)s * sizeof(int) + (size_t)n;
+  return dbl * sizeof(double) + ((tail + 7) & ~(size_t)7);
+}
+
 __global__ void __launch_bounds__(kSolveWarps * 32)
 decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, int n, int s,
                     const double *__restrict__ a0, const double *__restrict__ Nmat, const double *__restrict__ coef,
                     double *__restrict__ a_out, double *__restrict__ resid_out, double *maxres) {
-  __shared__ double M[kSolveWarps][NGC_MAX_S][NGC_MAX_S + 1];
-  __shared__ double zs[kSolveWarps][NGC_MAX_S];
-  __shared__ double as[kSolveWarps][NGC_MAX_N];
-  __shared__ int tlist[kSolveWarps][NGC_MAX_S];
-  __shared__ unsigned char used[kSolveWarps][NGC_MAX_N];
-
+  extern __shared__ __align__(16) unsigned char solve_smem[];
+  const int warps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int b = blockIdx.x * kSolveWarps + w;
+  const int b = blockIdx.x * warps + w;
   if (b >= batch) return;
+  const int ldm = s + 1;
+  double *M = reinterpret_cast<double *>(solve_smem + (size_t)w * solve_warp_bytes(n, s));  // [s][s+1]
+  double *zs = M + (size_t)s * ldm;
+  double *as = zs + s;
+  int *tlist = reinterpret_cast<int *>(as + n);
+  unsigned char *used = reinterpret_cast<unsigned char *>(tlist + s);
   uint64_t m0, m1;
   if (masks) { m0 = masks[2 * b]; m1 = masks[2 * b + 1]; }
   else { m0 = one.w[0]; m1 = one.w[1]; }
@@ -38,22 +49,22 @@ decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, 
     int kept = 0, nt = 0;
     for (int i = 0; i < n; ++i) {
       const bool in = ((i < 64 ? (m0 >> i) : (m1 >> (i - 64))) & 1ull) != 0;
-      if (in && kept < n - s) { used[w][i] = 1; ++kept; }
-      else { used[w][i] = 0; if (nt < s) tlist[w][nt] = i; ++nt; }
+      if (in && kept < n - s) { used[i] = 1; ++kept; }
+      else { used[i] = 0; if (nt < s) tlist[nt] = i; ++nt; }
     }
   }
   __syncwarp();
 
   if (s > 0) {
     if (lane < s) {
-      const int row = tlist[w][lane];
-      for (int c = 0; c < s; ++c) M[w][lane][c] = Nmat[(size_t)row * s + c];
-      M[w][lane][s] = -a0[row];
+      const int row = tlist[lane];
+      for (int c = 0; c < s; ++c) M[(lane) * ldm + (c)] = Nmat[(size_t)row * s + c];
+      M[(lane) * ldm + (s)] = -a0[row];
     }
     __syncwarp();
     for (int p = 0; p < s; ++p) {
       // pivot: largest magnitude in column p among rows >= p, smallest row on ties
-      double v = (lane >= p && lane < s) ? fabs(M[w][lane][p]) : -1.0;
+      double v = (lane >= p && lane < s) ? fabs(M[(lane) * ldm + (p)]) : -1.0;
       int q = lane;
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) {
@@ -63,32 +74,32 @@ decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, 
       }
       if (q != p) {
         for (int c = lane; c <= s; c += 32) {
-          const double tmp = M[w][p][c];
-          M[w][p][c] = M[w][q][c];
-          M[w][q][c] = tmp;
+          const double tmp = M[(p) * ldm + (c)];
+          M[(p) * ldm + (c)] = M[(q) * ldm + (c)];
+          M[(q) * ldm + (c)] = tmp;
         }
       }
       __syncwarp();
       if (lane > p && lane < s) {
-        const double f = M[w][lane][p] / M[w][p][p];
-        for (int c = p + 1; c <= s; ++c) M[w][lane][c] -= f * M[w][p][c];
+        const double f = M[(lane) * ldm + (p)] / M[(p) * ldm + (p)];
+        for (int c = p + 1; c <= s; ++c) M[(lane) * ldm + (c)] -= f * M[(p) * ldm + (c)];
       }
       __syncwarp();
     }
     for (int p = s - 1; p >= 0; --p) {      // column-oriented back substitution
-      if (lane == p) zs[w][p] = M[w][p][s] / M[w][p][p];
+      if (lane == p) zs[p] = M[(p) * ldm + (s)] / M[(p) * ldm + (p)];
       __syncwarp();
-      if (lane < p) M[w][lane][s] -= M[w][lane][p] * zs[w][p];
+      if (lane < p) M[(lane) * ldm + (s)] -= M[(lane) * ldm + (p)] * zs[p];
       __syncwarp();
     }
   }
   for (int i = lane; i < n; i += 32) {
     double v = 0.0;
-    if (used[w][i]) {
+    if (used[i]) {
       v = a0[i];
-      for (int c = 0; c < s; ++c) v += Nmat[(size_t)i * s + c] * zs[w][c];
+      for (int c = 0; c < s; ++c) v += Nmat[(size_t)i * s + c] * zs[c];
     }
-    as[w][i] = v;
+    as[i] = v;
     a_out[(size_t)b * n + i] = v;
   }
   __syncwarp();
@@ -99,7 +110,7 @@ decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, 
     for (int t = 0; t <= s; ++t) {
       int i = j - t;
       if (i < 0) i += n;
-      acc += as[w][i] * coef[(size_t)i * (s + 1) + t];
+      acc += as[i] * coef[(size_t)i * (s + 1) + t];
     }
     const double r = fabs(acc - 1.0);
     worst = fmax(worst, isnan(r) ? (double)INFINITY : r);
@@ -183,9 +194,11 @@ cudaError_t launch_gd_update(float *theta, const float *grad, long long l, float
 cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *masks_dev, MaskArg one, int batch,
                                 double *a_dev, double *resid_dev, double *maxres_dev, cudaStream_t stream) {
   const ngc_level_t &lv = p.lv[layer];
-  const unsigned blocks = (unsigned)((batch + kSolveWarps - 1) / kSolveWarps);
-  decode_solve_kernel<<<blocks, kSolveWarps * 32, 0, stream>>>(masks_dev, one, batch, p.n, lv.s, lv.d_a0, lv.d_N,
-                                                              lv.d_coef, a_dev, resid_dev, maxres_dev);
+  const int warps = (batch < kSolveWarps) ? batch : kSolveWarps;
+  const unsigned blocks = (unsigned)((batch + warps - 1) / warps);
+  const size_t smem = (size_t)warps * solve_warp_bytes(p.n, lv.s);  // at most 4 x 10.3 KB
+  decode_solve_kernel<<<blocks, warps * 32, smem, stream>>>(masks_dev, one, batch, p.n, lv.s, lv.d_a0, lv.d_N,
+                                                           lv.d_coef, a_dev, resid_dev, maxres_dev);
   return cudaGetLastError();
 }
 

@@ -48,6 +48,8 @@ cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_de
 
 // Same encode for long gradients (dense models): every partial gradient is read once, windows live in
 // registers.  ws is [group][slot][ld_ws] fp32, ld_ws a multiple of 4 and >= d.
+// True when an SM that holds a CTA of the gradient kernel chosen for `m` can still take a one-warp block.
+bool gemv_pair_leaves_room(const ngc_model_t &m);
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
                                int s, long long d, void *coded, int coded_dtype, cudaStream_t stream);
 

@@ -328,8 +328,18 @@ cudaError_t launch_one(const GemvParams &p, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+// Whether one more small block (a warp or two, a few KB of shared memory) still fits on an SM that
+// holds a CTA of this kernel: registers are what runs out first (512 threads x 128 registers fill the file).
+template <typename XT, int VPT, int R, int ACT>
+bool room_beside(const GemvParams &p) {
+  cudaFuncAttributes attr;
+  if (cudaFuncGetAttributes(&attr, gemv_pair_kernel<XT, VPT, R, ACT>) != cudaSuccess) return false;
+  const size_t smem = (size_t)p.stages * p.stage_bytes + kSmemReserve;
+  return (size_t)attr.numRegs * kThreads + 64 * 64 <= 65536 && smem + 16384 <= 233472;
+}
+
 template <typename XT, int ACT>
-cudaError_t launch_shape(GemvParams &p, cudaStream_t stream) {
+cudaError_t launch_shape(GemvParams &p, cudaStream_t stream, bool *room = nullptr) {
   const int nv = p.d / Vec<XT>::N;
   int vpt = (nv + kThreads - 1) / kThreads;
   int R;
@@ -342,6 +352,10 @@ cudaError_t launch_shape(GemvParams &p, cudaStream_t stream) {
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
+  if (room) {  // query only, nothing is launched
+    *room = (vpt == 1) ? room_beside<XT, 1, 8, ACT>(p) : (vpt == 2) ? room_beside<XT, 2, 4, ACT>(p) : room_beside<XT, 4, 2, ACT>(p);
+    return cudaSuccess;
+  }
   if (vpt == 1) return launch_one<XT, 1, 8, ACT>(p, stream);
   if (vpt == 2) return launch_one<XT, 2, 4, ACT>(p, stream);
   return launch_one<XT, 4, 2, ACT>(p, stream);
@@ -380,6 +394,18 @@ cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const 
   }
   p.row_bytes = m.d * 2;
   return act ? launch_shape<__nv_bfloat16, 1>(p, stream) : launch_shape<__nv_bfloat16, 0>(p, stream);
+}
+
+bool gemv_pair_leaves_room(const ngc_model_t &m) {
+  GemvParams p;
+  p.d = m.d;
+  p.row_bytes = m.d * (m.x_dtype == NGC_F32 ? 4 : 2);
+  const int act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
+  bool room = false;
+  cudaError_t e;
+  if (m.x_dtype == NGC_F32) e = act ? launch_shape<float, 1>(p, 0, &room) : launch_shape<float, 0>(p, 0, &room);
+  else e = act ? launch_shape<__nv_bfloat16, 1>(p, 0, &room) : launch_shape<__nv_bfloat16, 0>(p, 0, &room);
+  return e == cudaSuccess && room;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -445,49 +471,99 @@ combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const 
 }  // namespace
 
 namespace {
-// Encode for long gradients (dense models, one scratch slot per group): every thread owns 2 columns
-// and walks all n workers, holding a ring of W partial gradients in registers exactly as loaded
-// (fp32): s+1 of them form the worker's window, the other W-s-1 slots are loads still in flight for
-// the workers to come, and nothing touches a slot before its turn.  The arithmetic is done in the
-// type of the coded gradients (fp32 products and sums for fp32 storage).  Each partial gradient is
-// read once and never staged in shared memory.
-template <typename CT, int W>
-__global__ void __launch_bounds__(256)
-encode_stream_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n, int s,
-                     long long d, CT *__restrict__ coded) {
-  const long long col = ((long long)blockIdx.x * 256 + threadIdx.x) * 2;
+// Encode for long gradients (dense models, one scratch slot per group): every thread owns 4 columns
+// and walks a contiguous chunk of the workers (blockIdx.y), holding a ring of W = S1 + LOOK partial
+// gradients in registers exactly as loaded (fp32): S1 = s+1 of them form the worker's window, the
+// other LOOK slots are loads in flight for the workers to come, and nothing touches a slot before its
+// turn.  The window length is a template parameter, so the inner loops carry no predicates; the
+// chunk's coefficients are converted to the coded type once per block into shared memory.  The
+// arithmetic is done in the type of the coded gradients (fp32 storage: packed fp32 fused
+// multiply-adds, two columns per instruction).  Inside a chunk each partial gradient is read once;
+// chunks overlap by s groups, which come from L2.
+constexpr int kEncLook = 6;
+constexpr int kEncMaxS1 = 12;
+
+template <typename CT, int S1>
+__global__ void __launch_bounds__(128)
+encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n,
+                     long long d, int chunk, CT *__restrict__ coded) {
+  constexpr int W = S1 + kEncLook;
+  __shared__ CT cs[NGC_MAX_N * S1];
+  const int first = blockIdx.y * chunk;
+  const int last = (first + chunk < n) ? first + chunk : n;  // workers first .. last-1
+  if (first >= last) return;
+  for (int e = threadIdx.x; e < (last - first) * S1; e += 128) cs[e] = (CT)coef[(size_t)first * S1 + e];
+  __syncthreads();
+  const long long col = ((long long)blockIdx.x * 128 + threadIdx.x) * 4;
   if (col >= d) return;
+  const int need = last - first + S1 - 1;  // groups first .. first+need-1 (mod n) are read by this chunk
   const float *src = ws + col;
-  float2 win[W];
+  ulonglong2 win[W];  // each half is a pair of consecutive fp32 columns
+  int next = first;   // group that the next free slot receives
+  int loaded = 0;
 #pragma unroll
-  for (int t = 0; t < W; ++t) win[t] = __ldg(reinterpret_cast<const float2 *>(src + (size_t)(t % n) * ld_ws));
-  const bool pair = (d % 2 == 0);
-  int next = W % n;  // group that the next freed slot receives
-  for (int i0 = 0; i0 < n; i0 += W) {
+  for (int t = 0; t < W; ++t) {
+    if (loaded < need) win[t] = __ldg(reinterpret_cast<const ulonglong2 *>(src + (size_t)next * ld_ws));
+    ++loaded;
+    if (++next == n) next = 0;
+  }
+  const int store_mode = (d % 4 == 0) ? 4 : (d % 2 == 0) ? 2 : 1;
+  const CT *ci = cs;
+  CT *dst = coded + (size_t)first * d + col;
+  for (int i0 = first; i0 < last; i0 += W) {
 #pragma unroll
     for (int t = 0; t < W; ++t) {
-      const int i = i0 + t;
-      if (i < n) {
-        CT acc0 = 0, acc1 = 0;
-        const double *ci = coef + (size_t)i * (s + 1);
+      if (i0 + t < last) {
+        CT out[4];
+        if constexpr (sizeof(CT) == 4) {
+          f32x2 a01 = 0ull, a23 = 0ull;
 #pragma unroll
-        for (int k = 0; k < W; ++k) {
-          if (k <= s) {
-            const CT c = (CT)__ldg(ci + k);
-            acc0 = fma(c, (CT)win[(t + k) % W].x, acc0);
-            acc1 = fma(c, (CT)win[(t + k) % W].y, acc1);
+          for (int k = 0; k < S1; ++k) {
+            const f32x2 cc = pack2(ci[k], ci[k]);
+            fma2(a01, cc, win[(t + k) % W].x);
+            fma2(a23, cc, win[(t + k) % W].y);
+          }
+          unpack2(a01, out[0], out[1]);
+          unpack2(a23, out[2], out[3]);
+        } else {
+          out[0] = out[1] = out[2] = out[3] = 0;
+#pragma unroll
+          for (int k = 0; k < S1; ++k) {
+            float g0, g1, g2, g3;
+            unpack2(win[(t + k) % W].x, g0, g1);
+            unpack2(win[(t + k) % W].y, g2, g3);
+            out[0] = fma(ci[k], (CT)g0, out[0]);
+            out[1] = fma(ci[k], (CT)g1, out[1]);
+            out[2] = fma(ci[k], (CT)g2, out[2]);
+            out[3] = fma(ci[k], (CT)g3, out[3]);
           }
         }
-        CT *dst = coded + (size_t)i * d + col;
-        if (pair) {
-          if (sizeof(CT) == 8) *reinterpret_cast<double2 *>(dst) = make_double2((double)acc0, (double)acc1);
-          else *reinterpret_cast<float2 *>(dst) = make_float2((float)acc0, (float)acc1);
+        if (store_mode == 4) {
+          if constexpr (sizeof(CT) == 8) {
+            reinterpret_cast<double2 *>(dst)[0] = make_double2((double)out[0], (double)out[1]);
+            reinterpret_cast<double2 *>(dst)[1] = make_double2((double)out[2], (double)out[3]);
+          } else {
+            *reinterpret_cast<float4 *>(dst) = make_float4((float)out[0], (float)out[1], (float)out[2], (float)out[3]);
+          }
+        } else if (store_mode == 2) {
+          if constexpr (sizeof(CT) == 8) {
+            reinterpret_cast<double2 *>(dst)[0] = make_double2((double)out[0], (double)out[1]);
+            if (col + 2 < d) reinterpret_cast<double2 *>(dst)[1] = make_double2((double)out[2], (double)out[3]);
+          } else {
+            reinterpret_cast<float2 *>(dst)[0] = make_float2((float)out[0], (float)out[1]);
+            if (col + 2 < d) reinterpret_cast<float2 *>(dst)[1] = make_float2((float)out[2], (float)out[3]);
+          }
         } else {
-          dst[0] = acc0;
-          if (col + 1 < d) dst[1] = acc1;
+          dst[0] = out[0];
+          if (col + 1 < d) dst[1] = out[1];
+          if (col + 2 < d) dst[2] = out[2];
+          if (col + 3 < d) dst[3] = out[3];
         }
-        // group i is no longer needed; its slot takes group i + W
-        win[t] = __ldg(reinterpret_cast<const float2 *>(src + (size_t)next * ld_ws));
+        ci += S1;
+        dst += d;
+        // the oldest group is no longer needed; its slot takes the next group of the chunk, if any is left
+        if (loaded < need) win[t] = __ldg(reinterpret_cast<const ulonglong2 *>(src + (size_t)next * ld_ws));
+        ++loaded;
         if (++next == n) next = 0;
       }
     }
@@ -516,14 +592,53 @@ encode_simple_kernel(const RowSplit split, const float *__restrict__ ws, long lo
 }
 
 template <typename CT>
+using EncodeKernel = void (*)(const float *, long long, const double *, int, long long, int, CT *);
+
+template <typename CT>
+EncodeKernel<CT> encode_window_for(int s1) {
+  switch (s1) {
+    case 1: return encode_window_kernel<CT, 1>;
+    case 2: return encode_window_kernel<CT, 2>;
+    case 3: return encode_window_kernel<CT, 3>;
+    case 4: return encode_window_kernel<CT, 4>;
+    case 5: return encode_window_kernel<CT, 5>;
+    case 6: return encode_window_kernel<CT, 6>;
+    case 7: return encode_window_kernel<CT, 7>;
+    case 8: return encode_window_kernel<CT, 8>;
+    case 9: return encode_window_kernel<CT, 9>;
+    case 10: return encode_window_kernel<CT, 10>;
+    case 11: return encode_window_kernel<CT, 11>;
+    case 12: return encode_window_kernel<CT, 12>;
+    default: return nullptr;
+  }
+}
+
+template <typename CT>
 cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long ld_ws, const double *coef, int n, int s,
                               long long d, CT *coded, cudaStream_t stream) {
-  const unsigned blocks = (unsigned)((d + 511) / 512);
-  // ring size = window (s+1) plus at least two slots of loads in flight; one scratch slot per group only
-  if (split.P == 1 && s + 1 <= 2) encode_stream_kernel<CT, 4><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
-  else if (split.P == 1 && s + 1 <= 6) encode_stream_kernel<CT, 8><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
-  else if (split.P == 1 && s + 1 <= 12) encode_stream_kernel<CT, 16><<<blocks, 256, 0, stream>>>(ws, ld_ws, coef, n, s, d, coded);
-  else encode_simple_kernel<CT><<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
+  EncodeKernel<CT> kern = (split.P == 1 && s + 1 <= kEncMaxS1) ? encode_window_for<CT>(s + 1) : nullptr;
+  if (!kern) {
+    encode_simple_kernel<CT><<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
+    return cudaGetLastError();
+  }
+  // Number of worker chunks: the blocks run in rounds of `capacity` resident blocks, a block's time grows
+  // with the groups it reads (chunk + s) plus a fixed part; take the split with the least rounds x time.
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 128, 0);
+  if (e != cudaSuccess) return e;
+  const long long capacity = (long long)(per_sm > 0 ? per_sm : 1) * device_sm_count();
+  const long long col_blocks = (d + 511) / 512;
+  int best_chunks = 1;
+  long long best_cost = -1;
+  for (int chunks = 1; chunks <= n && chunks <= 16; ++chunks) {
+    const int chunk = (n + chunks - 1) / chunks;
+    const long long blocks = col_blocks * ((n + chunk - 1) / chunk);
+    const long long cost = ((blocks + capacity - 1) / capacity) * (chunk + s + 4);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_chunks = chunks; }
+  }
+  const int chunk = (n + best_chunks - 1) / best_chunks;
+  const dim3 grid((unsigned)col_blocks, (unsigned)((n + chunk - 1) / chunk));
+  kern<<<grid, 128, 0, stream>>>(ws, ld_ws, coef, n, d, chunk, coded);
   return cudaGetLastError();
 }
 }  // namespace

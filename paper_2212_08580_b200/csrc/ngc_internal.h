@@ -36,6 +36,12 @@ struct ngc_plan_s {
   int a_batch_cap = 0;
   int *d_status = nullptr;     // [0] timeout flag, [1] scratch
   double *d_maxres = nullptr;  // largest residual seen by asynchronous decodes
+  // ngc_step solves the decoding vector on a stream of its own while the gradients are computed
+  void *side_stream = nullptr; // cudaStream_t, non-blocking
+  void *ev_solved = nullptr;   // cudaEvent_t: d_a holds the vector of the current step
+  void *ev_decoded = nullptr;  // cudaEvent_t: the last decode has read d_a
+  int overlap_kind = -1, overlap_d = -1, overlap_dtype = -1;  // model the answer below was taken for
+  bool overlap_ok = false;     // the gradient kernel leaves room for the solve's warp on its SMs
   // staging for ngc_step_host
   void *st_X = nullptr, *st_y = nullptr, *st_theta = nullptr, *st_coded = nullptr, *st_grad = nullptr;
   size_t st_X_bytes = 0, st_y_bytes = 0, st_theta_bytes = 0, st_coded_bytes = 0, st_grad_bytes = 0;
