@@ -170,8 +170,63 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__rest
   }
 }
 
+// The same reduction for long gradients, where there are enough columns to fill the GPU without splitting
+// the rows: one thread owns V consecutive parameters and walks the rows with a non-zero weight in
+// index order (a compacted list in shared memory), several loads in flight, no exchange between threads.
+template <typename CT, int V>
+__global__ void __launch_bounds__(256) decode_flat_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
+                                                          int n, long long l, float *__restrict__ grad) {
+  __shared__ double as[NGC_MAX_N];
+  __shared__ double wt[NGC_MAX_N];
+  __shared__ int row[NGC_MAX_N];
+  __shared__ int count;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) as[i] = a[i];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int m = 0;
+    for (int i = 0; i < n; ++i)
+      if (as[i] != 0.0) { wt[m] = as[i]; row[m] = i; ++m; }
+    count = m;
+  }
+  __syncthreads();
+  const long long col = ((long long)blockIdx.x * 256 + threadIdx.x) * V;
+  if (col >= l) return;
+  const int m = count;
+  double acc[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) acc[e] = 0.0;
+#pragma unroll 8
+  for (int t = 0; t < m; ++t) {
+    const CT *src = coded + (size_t)row[t] * l + col;
+    alignas(16) CT v[V];
+    if (V * sizeof(CT) == 16) *reinterpret_cast<uint4 *>(v) = __ldg(reinterpret_cast<const uint4 *>(src));
+    else if (V * sizeof(CT) == 8) *reinterpret_cast<uint2 *>(v) = __ldg(reinterpret_cast<const uint2 *>(src));
+    else v[0] = __ldg(src);
+    const double w = wt[t];
+#pragma unroll
+    for (int e = 0; e < V; ++e) acc[e] = fma(w, (double)v[e], acc[e]);
+  }
+  float *dst = grad + col;
+  if (V == 4 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+    *reinterpret_cast<float4 *>(dst) = make_float4((float)acc[0], (float)acc[V > 1 ? 1 : 0], (float)acc[V > 2 ? 2 : 0], (float)acc[V > 3 ? 3 : 0]);
+  } else if (V == 2 && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+    *reinterpret_cast<float2 *>(dst) = make_float2((float)acc[0], (float)acc[V > 1 ? 1 : 0]);
+  } else {
+#pragma unroll
+    for (int e = 0; e < V; ++e) dst[e] = (float)acc[e];
+  }
+}
+
+constexpr long long kDecodeFlatFrom = 1 << 16;  // parameters from which one thread per V columns fills the GPU
+
 template <typename CT, int V>
 cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, cudaStream_t stream) {
+  if (l >= kDecodeFlatFrom) {
+    const long long per_block = 256 * V;
+    decode_flat_kernel<CT, V><<<(unsigned)((l + per_block - 1) / per_block), 256, 0, stream>>>(
+        static_cast<const CT *>(coded), a, n, l, grad);
+    return cudaGetLastError();
+  }
   const long long per_block = 32 * V;
   const unsigned blocks = (unsigned)((l + per_block - 1) / per_block);
   decode_kernel<CT, V><<<blocks, kDecWarps * 32, 0, stream>>>(static_cast<const CT *>(coded), a, n, l, grad);

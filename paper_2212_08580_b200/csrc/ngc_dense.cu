@@ -51,6 +51,8 @@ struct FwdParams {
 // D[M x N] = A^T B per batch, A stored [batch][K][M] and B stored [batch][K][N_total] (both row-major bf16,
 // read as M/N-major operands).  Tile = (batch j, 128 rows of M, 256 columns of N_total).  Batches are taken
 // last to first: the forward pass that ran just before went first to last, so its last batches are still in L2.
+// The single-CTA kernel numbers its tiles M-block-major: a ragged last M block (the bias row of an MLP layer)
+// is then what the CTAs of a second round get, not a full tile.
 struct TnParams {
   int batch, m_tiles, n_tiles, num_tiles;
   int num_k;      // K chunks of 64
@@ -741,7 +743,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t ph = 0;
       const uint32_t tx = (uint32_t)(2 + p.nbox) * 8192u;
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = p.batch - 1 - tile / (p.n_tiles * p.m_tiles);
+        const int nt = tile % p.n_tiles, j = p.batch - 1 - (tile / p.n_tiles) % p.batch, mt = tile / (p.n_tiles * p.batch);
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
           mbar_expect_tx(s.full[st], tx);
@@ -787,7 +789,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t aph = 0;
     const bool vec = (p.out_ld % 4 == 0) && (p.n_store % 4 == 0) && (p.out_batch % 4 == 0);
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = p.batch - 1 - tile / (p.n_tiles * p.m_tiles);
+      const int nt = tile % p.n_tiles, j = p.batch - 1 - (tile / p.n_tiles) % p.batch, mt = tile / (p.n_tiles * p.batch);
       if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
       tc_fence_after();
       const int m = mt * 128 + q * 32 + lane;
