@@ -230,7 +230,7 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     ngc::RowSplit split;
     split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
     NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, ngc_num_params(m), coded, cdt, stream));
-    p->launches += (h % 64 == 0) ? 8 : 7;  // convert, transpose, forward, (W2 layouts,) head, 2 backward, encode
+    p->launches += ngc::mlp_launch_count(h);
     return NGC_OK;
   }
   return NGC_ERR_INVALID;

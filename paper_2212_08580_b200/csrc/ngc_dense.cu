@@ -513,28 +513,42 @@ mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C
 
 // ------------------------------------------------------------------------------------------------
 // MLP head on the tensor cores (hidden a multiple of 64, at most 512; at most 16 classes).  Per tile of
-// 128 samples, everything stays in shared / tensor memory:
-//   1. TMA brings the 128 x hidden tile of h (bf16, K-major, 128-byte swizzle);
+// 128 samples of one partition, everything stays in shared / tensor memory:
+//   1. TMA brings the 128 x hidden tile of h (bf16, K-major, 128-byte swizzle), in groups of four 64-column chunks;
 //   2. z[128 x 16] = h W2 (W2^T resident in shared memory as the B operand, N = 16);
-//   3. one thread per sample: z + b2 -> softmax -> delta2; delta2 goes to global memory (for dW2) and, as
-//      a bf16 row of a swizzled 128 x 64 tile, becomes the A operand of the next contraction;
-//   4. (delta2 W2^T)[128 x hidden] with K = 16: one MMA per 256 hidden units;
-//   5. the threads mask by h > 0 (read from the tile in its swizzled layout), overwrite h by delta1 in
-//      place, and TMA stores the tile to delta1[rows][hidden].
+//   3. one thread per sample: z + b2 -> softmax -> delta2, which, as a bf16 row of a swizzled 128 x 64 tile,
+//      becomes an operand of the next contractions;
+//   4. hidden a multiple of 128: dW2 += h^T delta2 (samples as K: both tiles read M/N-major), accumulated in
+//      tensor memory over the CTA's tiles of a partition; db2 by warp shuffles.  Otherwise delta2 goes to
+//      global memory and a backward contraction forms dW2;
+//   5. (delta2 W2^T)[128 x hidden] with K = 16: one MMA per 256 hidden units;
+//   6. the threads mask by h > 0 (read from the tile in its swizzled layout) and overwrite h by delta1 in
+//      place; the producer stores each finished group to delta1[rows][hidden] and reloads it with the next
+//      tile's h while the other group is still being worked on.
 // ------------------------------------------------------------------------------------------------
-constexpr int kHeadTcThreads = 192;
+constexpr int kHeadEpiThreads = 512;  // 16 epilogue warps: four per tensor-memory quadrant
+constexpr int kHeadTcThreads = 64 + kHeadEpiThreads;  // + producer and MMA warps
+__device__ __forceinline__ void head_epi_sync() { asm volatile("bar.sync 6, %0;" ::"n"(kHeadEpiThreads) : "memory"); }
 
 struct HeadTcParams {
-  int hidden, C, num_tiles;
+  int hidden, C, rows, tiles_per_part, num_tiles;  // a tile = 128 rows of one partition
   const float *b2;
   const int *y;
-  long long rows_total;
-  __nv_bfloat16 *D2;  // [rows_total][64]
+  __nv_bfloat16 *D2;  // [k * rows][64]: delta2 rows, written only when the output-layer gradient is formed elsewhere
+  int fuse;           // 1: [dW2; db2] = [h 1]^T delta2 is formed here (hidden a multiple of 128)
+  float *slots;       // [k][max_slots][hidden * C + C]: partial sums of the CTAs that share a partition
+  int max_slots;
+  int *counters;      // [k], zero at launch: CTAs that have delivered their slot of a partition
+  float *G;           // [dW2; db2] of partition j goes to G + j * g_batch
+  size_t g_batch;
   int *status;
 };
 
+// Tiles [begin, end) of CTA c when `tiles` tiles are cut into `grid` contiguous ranges.
+__host__ __device__ inline int head_tile_begin(int c, int tiles, int grid) { return (int)((long long)c * tiles / grid); }
+
 __global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, __nv_bfloat16 *__restrict__ W2t,
-                               __nv_bfloat16 *__restrict__ W2k) {
+                               __nv_bfloat16 *__restrict__ W2k, int *__restrict__ counters, int k) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < 16 * hidden) {  // W2t[c][hc]
     const int c = i / hidden, hc = i % hidden;
@@ -544,6 +558,7 @@ __global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, 
     const int hc = i / 64, c = i % 64;
     W2k[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
   }
+  if (i < k) counters[i] = 0;
 }
 
 __global__ void __launch_bounds__(kHeadTcThreads, 1)
@@ -553,26 +568,39 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char *sm = smem_raw + ((1024u - (base & 1023u)) & 1023u);
-  const int nchunk = p.hidden / 64, nhalf = (p.hidden + 255) / 256;
+  const int nchunk = p.hidden / 64, nhalf = (p.hidden + 255) / 256, ngroups = (nchunk + 1) / 2;
   unsigned char *htile = sm;                                  // nchunk x [128 x 64] bf16
   unsigned char *d2tile = htile + (size_t)nchunk * 16384;     // [128 x 64] bf16 (16 columns used)
   unsigned char *w2k = d2tile + 16384;                        // nhalf x [256 x 64] bf16
   unsigned char *w2t = w2k + (size_t)nhalf * 32768;           // nchunk x [16 x 64] bf16
   uint64_t *bars = reinterpret_cast<uint64_t *>(w2t + (size_t)nchunk * 2048);
-  const uint32_t h_full = smem_u32(&bars[0]), h_empty = smem_u32(&bars[1]), z_full = smem_u32(&bars[2]),
-                 d2_full = smem_u32(&bars[3]), d_full = smem_u32(&bars[4]), d_empty = smem_u32(&bars[5]),
-                 w_full = smem_u32(&bars[6]);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[7]);
-  float *b2s = reinterpret_cast<float *>(&bars[8]);           // 16 floats
+  // The tile lives in shared memory as groups of two 64-column chunks.  Group g is loaded (h), consumed,
+  // overwritten in place (delta1), stored and reloaded with the next tile's h on its own barriers, so the
+  // memory traffic of the finished groups hides behind the arithmetic on the others.
+  uint32_t h_full[4], m_done[4];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    h_full[g] = smem_u32(&bars[g]);
+    m_done[g] = smem_u32(&bars[4 + g]);
+  }
+  const uint32_t z_full = smem_u32(&bars[8]), d2_full = smem_u32(&bars[9]), d_full = smem_u32(&bars[10]),
+                 d_empty = smem_u32(&bars[11]), w_full = smem_u32(&bars[12]);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[13]);
+  float *b2s = reinterpret_cast<float *>(&bars[14]);          // 16 floats
+  float *dbx = reinterpret_cast<float *>(&bars[22]);          // [4 quadrants][16]: bias-gradient partial sums
+  volatile int *last_flag = reinterpret_cast<volatile int *>(&bars[54]);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(h_full, 1);
-    mbar_init(h_empty, 1);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      mbar_init(h_full[g], 1);
+      mbar_init(m_done[g], kHeadEpiThreads);
+    }
     mbar_init(z_full, 1);
     mbar_init(d2_full, 128);
     mbar_init(d_full, 1);
-    mbar_init(d_empty, 128);
+    mbar_init(d_empty, kHeadEpiThreads);
     mbar_init(w_full, 1);
     mbar_fence_init();
   }
@@ -582,47 +610,83 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t z_acc = tmem_base, d_acc = tmem_base + 256u;
+  const uint32_t z_acc = tmem_base, w2_acc = tmem_base + 32u, d_acc = tmem_base + 256u;
   bool failed = false;
+  const int grid = (int)gridDim.x, tpp = p.tiles_per_part;
+  const int t_begin = head_tile_begin((int)blockIdx.x, p.num_tiles, grid),
+            t_end = head_tile_begin((int)blockIdx.x + 1, p.num_tiles, grid);
 
   if (warp == 0) {
     if (lane == 0) {
       mbar_expect_tx(w_full, (uint32_t)(nchunk * 2048 + nhalf * 32768));
       for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(w2t + kc * 2048), &tmW2t, kc * 64, 0, w_full);
       for (int hh = 0; hh < nhalf; ++hh) tma_load_2d(smem_u32(w2k + hh * 32768), &tmW2k, 0, hh * 256, w_full);
+      auto load_group = [&](int tile, int g) {
+        const int j = tile / tpp, rb = tile % tpp, c0 = g * 2, c1 = min(nchunk, c0 + 2);
+        mbar_expect_tx(h_full[g], (uint32_t)(c1 - c0) * 16384u);
+        for (int kc = c0; kc < c1; ++kc)
+          tma_load_3d(smem_u32(htile + kc * 16384), &tmH, kc * 64, rb * 128, j, h_full[g]);
+      };
+      for (int g = 0; g < ngroups; ++g) load_group(t_begin, g);
       uint32_t ph = 0;
-      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        if (!mbar_wait(h_empty, ph ^ 1u)) { failed = true; break; }
-        mbar_expect_tx(h_full, (uint32_t)nchunk * 16384u);
-        for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(htile + kc * 16384), &tmH, kc * 64, tile * 128, h_full);
+      for (int tile = t_begin; tile < t_end && !failed; ++tile) {
+        const int j = tile / tpp, rb = tile % tpp;
+        for (int g = 0; g < ngroups; ++g) {
+          // delta1 has replaced h in group g: store it, and once the store has read shared memory bring the
+          // next tile's h into the same chunks
+          if (!mbar_wait(m_done[g], ph)) { failed = true; break; }
+          const int c0 = g * 2, c1 = min(nchunk, c0 + 2);
+          for (int kc = c0; kc < c1; ++kc) tma_store_3d(&tmD1, kc * 64, rb * 128, j, smem_u32(htile + kc * 16384));
+          tma_store_commit_and_wait_read();
+          if (tile + 1 < t_end) load_group(tile + 1, g);
+        }
         ph ^= 1u;
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc_z = instr_desc_bf16(128, 16, 0, 0);
+      const uint32_t idesc_z = instr_desc_bf16(128, 16, 0, 0), idesc_w = instr_desc_bf16(128, 16, 1, 1);
+      const int nmb = p.hidden / 128;
       uint32_t ph = 0, dph = 0;
       if (!mbar_wait(w_full, 0)) failed = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        if (!mbar_wait(h_full, ph)) { failed = true; break; }
-        tc_fence_after();
-        for (int kc = 0; kc < nchunk; ++kc) {
-          const uint64_t ad = smem_desc_sw128(smem_u32(htile + kc * 16384), 16, 1024);
-          const uint64_t bd = smem_desc_sw128(smem_u32(w2t + kc * 2048), 16, 1024);
+      for (int tile = t_begin; tile < t_end && !failed; ++tile) {
+        for (int g = 0; g < ngroups && !failed; ++g) {
+          if (!mbar_wait(h_full[g], ph)) { failed = true; break; }
+          tc_fence_after();
+          for (int kc = g * 2; kc < min(nchunk, g * 2 + 2); ++kc) {
+            const uint64_t ad = smem_desc_sw128(smem_u32(htile + kc * 16384), 16, 1024);
+            const uint64_t bd = smem_desc_sw128(smem_u32(w2t + kc * 2048), 16, 1024);
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            mma_bf16(z_acc, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc_z, (kc | k4) != 0);
+            for (int k4 = 0; k4 < 4; ++k4)
+              mma_bf16(z_acc, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc_z, (kc | k4) != 0);
+          }
         }
+        if (failed) break;
         mma_commit(z_full);
         if (!mbar_wait(d2_full, ph)) { failed = true; break; }
         tc_fence_after();
-        const uint64_t ad = smem_desc_sw128(smem_u32(d2tile), 16, 1024);
+        const bool first = tile == t_begin || tile % tpp == 0;  // first tile of its partition in this CTA
+        const uint64_t ad1 = smem_desc_sw128(smem_u32(d2tile), 16, 1024);      // delta2, K-major (K = classes)
+        const uint64_t bdw = smem_desc_sw128(smem_u32(d2tile), 16384, 1024);   // delta2, N-major (K = samples)
         for (int hh = 0; hh < nhalf; ++hh) {
+          if (p.fuse) {
+            // dW2 block (128 hidden units x 16 classes) += h_block^T delta2 for the blocks inside this half:
+            // both operands are read M/N-major from the tiles the other contractions use K-major.  Issued
+            // ahead of the half's delta1 contraction, whose commit therefore covers them too: h may be
+            // overwritten once d_full has fired.  The second half's share runs under the first mask pass.
+            for (int mb = hh * 2; mb < min(nmb, hh * 2 + 2); ++mb) {
+              const uint64_t adw = smem_desc_sw128(smem_u32(htile + mb * 32768), 16384, 1024);
+#pragma unroll
+              for (int k8 = 0; k8 < 8; ++k8)  // 16 samples = 2048 bytes per instruction
+                mma_bf16(w2_acc + (uint32_t)mb * 16u, adw + (uint64_t)(k8 * 128), bdw + (uint64_t)(k8 * 128), idesc_w,
+                         !(first && k8 == 0));
+            }
+          }
           if (!mbar_wait(d_empty, dph ^ 1u)) { failed = true; break; }
           tc_fence_after();
           const int nh = min(256, p.hidden - hh * 256);
           const uint64_t bd = smem_desc_sw128(smem_u32(w2k + hh * 32768), 16, 1024);
-          mma_bf16(d_acc, ad, bd, instr_desc_bf16(128, nh, 0, 0), 0);  // K = 16: the 16 class columns
+          mma_bf16(d_acc, ad1, bd, instr_desc_bf16(128, nh, 0, 0), 0);  // K = 16: the 16 class columns
           mma_commit(d_full);
           dph ^= 1u;
         }
@@ -631,93 +695,162 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
     }
   } else {
     const int q = warp & 3, r = q * 32 + lane;  // row of the tile = tensor-memory lane
+    const int part = (warp - 2) >> 2;           // the four warps of a quadrant split every chunk: 16 columns each
+    const int tid_epi = (int)threadIdx.x - 64;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;  // row r inside a swizzled tile
     const uint32_t rx = (uint32_t)(r & 7);
+    const int wstride = p.hidden * p.C + p.C;
     uint32_t ph = 0, dph = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      const long long row = (long long)tile * 128 + r;
-      const bool valid = row < p.rows_total;
-      if (!mbar_wait(z_full, ph)) { failed = true; break; }
-      tc_fence_after();
-      float v[32];
-      tmem_ld32(z_acc + lane_off, v);
-      const int label = valid ? p.y[row] : -1;
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        v[c] += b2s[c];
-        if (c < p.C) mx = fmaxf(mx, v[c]);
-      }
-      float sum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        v[c] = c < p.C ? __expf(v[c] - mx) : 0.f;
-        sum += v[c];
-      }
-      const float inv = 1.f / sum;
-      uint32_t w[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float lo = (2 * u < p.C) ? v[2 * u] * inv - (2 * u == label ? 1.f : 0.f) : 0.f;
-        const float hi = (2 * u + 1 < p.C) ? v[2 * u + 1] * inv - (2 * u + 1 == label ? 1.f : 0.f) : 0.f;
-        const __nv_bfloat162 b2v = __floats2bfloat162_rn(lo, hi);
-        w[u] = *reinterpret_cast<const uint32_t *>(&b2v);
-      }
-      if (valid) {
-        uint4 *d2 = reinterpret_cast<uint4 *>(p.D2 + row * 64);
-        d2[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        d2[1] = make_uint4(w[4], w[5], w[6], w[7]);
-      }
-      *reinterpret_cast<uint4 *>(d2tile + row_off + ((0u ^ rx) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4 *>(d2tile + row_off + ((1u ^ rx) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-      fence_async_smem();
-      mbar_arrive(d2_full);
-      // the threads read h themselves below: observe the completion of its TMA copies directly
-      if (!mbar_wait(h_full, ph)) { failed = true; break; }
-      for (int hh = 0; hh < nhalf; ++hh) {
-        if (!mbar_wait(d_full, dph)) { failed = true; break; }
+    float db2_acc = 0.f;  // lane c of a part-0 warp: sum of delta2[., c] over the warp's rows
+    for (int tile = t_begin; tile < t_end; ++tile) {
+      const int j = tile / tpp, rb = tile % tpp;
+      const int prow = rb * 128 + r;
+      const bool valid = prow < p.rows;
+      const long long row = (long long)j * p.rows + prow;
+      if (part == 0) {
+        if (!mbar_wait(z_full, ph)) { failed = true; break; }
         tc_fence_after();
-        const int nh = min(256, p.hidden - hh * 256);
-        for (int gulp = 0; gulp * 128 < nh; ++gulp) {
-          uint32_t rr[128];
-          const int nch = min(4, (nh - gulp * 128) / 32);
-          tmem_ld_chunks<4>(d_acc + lane_off + gulp * 128, nch, rr);
-          if ((gulp + 1) * 128 >= nh) {  // the accumulator has been read completely
-            tc_fence_before();
-            mbar_arrive(d_empty);
-          }
+        float v[16];
+        tmem_ld16(z_acc + lane_off, v);
+        const int label = valid ? p.y[row] : -1;
+        float mx = -INFINITY;
 #pragma unroll
-          for (int g = 0; g < 16; ++g) {
-            if (g * 8 < nch * 32) {
-              const int col = hh * 256 + gulp * 128 + g * 8;  // hidden unit of the first of 8 values
-              unsigned char *hp = htile + (size_t)(col >> 6) * 16384 + row_off + ((((uint32_t)(col & 63) >> 3) ^ rx) << 4);
-              const uint4 hv = *reinterpret_cast<const uint4 *>(hp);
-              const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+        for (int c = 0; c < 16; ++c) {
+          v[c] += b2s[c];
+          if (c < p.C) mx = fmaxf(mx, v[c]);
+        }
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          v[c] = c < p.C ? __expf(v[c] - mx) : 0.f;
+          sum += v[c];
+        }
+        const float inv = valid ? 1.f / sum : 0.f;  // rows beyond the partition contribute nothing
+        uint32_t w[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float lo = (2 * u < p.C) ? v[2 * u] * inv - (2 * u == label ? 1.f : 0.f) : 0.f;
+          const float hi = (2 * u + 1 < p.C) ? v[2 * u + 1] * inv - (2 * u + 1 == label ? 1.f : 0.f) : 0.f;
+          const __nv_bfloat162 b2v = __floats2bfloat162_rn(lo, hi);
+          w[u] = *reinterpret_cast<const uint32_t *>(&b2v);
+        }
+        *reinterpret_cast<uint4 *>(d2tile + row_off + ((0u ^ rx) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4 *>(d2tile + row_off + ((1u ^ rx) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        fence_async_smem();
+        mbar_arrive(d2_full);
+        if (valid && !p.fuse) {
+          uint4 *d2 = reinterpret_cast<uint4 *>(p.D2 + row * 64);
+          d2[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          d2[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        if (p.fuse) {  // db2: column sums of the rounded delta2 over this warp's 32 rows, class c kept by lane c
+          float mine = 0.f;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            float t = __uint_as_float((c & 1) ? (w[c >> 1] & 0xffff0000u) : (w[c >> 1] << 16));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (lane == c) mine = t;
+          }
+          db2_acc += mine;
+        }
+      }
+      uint32_t rr[64];  // this thread's 16 columns of each of the (up to) four chunks of a 256-column half
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        if (g >= ngroups || failed) break;
+        // the threads read h themselves below: observe the completion of its TMA copies directly
+        if (!mbar_wait(h_full[g], ph)) { failed = true; break; }
+        if ((g & 1) == 0) {  // first group of a half: fetch the half's accumulator and hand it back at once
+          if (!mbar_wait(d_full, dph)) { failed = true; break; }
+          tc_fence_after();
+          const int hh = g >> 1, nlc = min(4, nchunk - hh * 4);
+#pragma unroll
+          for (int lc = 0; lc < 4; ++lc)
+            if (lc < nlc) tmem_ld16_nowait(d_acc + lane_off + (uint32_t)(lc * 64 + part * 16), &rr[lc * 16]);
+          tmem_ld_wait(rr);
+          tc_fence_before();
+          mbar_arrive(d_empty);
+          dph ^= 1u;
+        }
+        const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int kc = g * 2 + cc;  // chunk of 64 hidden units
+          if (kc < nchunk) {
+            unsigned char *crow = htile + (size_t)kc * 16384 + row_off;
+            uint4 hv[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              hv[i] = *reinterpret_cast<const uint4 *>(crow + ((((uint32_t)(part * 2 + i)) ^ rx) << 4));
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const uint32_t hw4[4] = {hv[i].x, hv[i].y, hv[i].z, hv[i].w};
               uint32_t o[4];
 #pragma unroll
               for (int t2 = 0; t2 < 4; ++t2) {
-                const float d0 = __uint_as_float(hw[t2] << 16) > 0.f ? __uint_as_float(rr[g * 8 + 2 * t2]) : 0.f;
-                const float d1 = __uint_as_float(hw[t2] & 0xffff0000u) > 0.f ? __uint_as_float(rr[g * 8 + 2 * t2 + 1]) : 0.f;
-                const __nv_bfloat162 db = __floats2bfloat162_rn(d0, d1);
-                o[t2] = *reinterpret_cast<const uint32_t *>(&db);
+                // (g & 1) * 2 + cc = chunk inside the half; delta1 = (h > 0) ? value : 0 as a bf16 pair
+                const int e = (((g & 1) * 2 + cc) * 16) + i * 8 + t2 * 2;
+                const __nv_bfloat162 dv = __floats2bfloat162_rn(__uint_as_float(rr[e]), __uint_as_float(rr[e + 1]));
+                const __nv_bfloat162 hb = *reinterpret_cast<const __nv_bfloat162 *>(&hw4[t2]);
+                const __nv_bfloat162 dm = __hmul2(dv, __hgt2(hb, zero2));
+                o[t2] = *reinterpret_cast<const uint32_t *>(&dm);
               }
-              *reinterpret_cast<uint4 *>(hp) = make_uint4(o[0], o[1], o[2], o[3]);
+              *reinterpret_cast<uint4 *>(crow + ((((uint32_t)(part * 2 + i)) ^ rx) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
           }
         }
-        dph ^= 1u;
+        fence_async_smem();
+        mbar_arrive(m_done[g]);  // this thread's share of delta1 sits where h was
       }
       if (failed) break;
-      // delta1 now sits where h was: hand the tile to TMA, then give the buffer back to the producer
-      fence_async_smem();
-      asm volatile("bar.sync 6, 128;" ::: "memory");
-      if (warp == 2 && lane == 0) {
-        for (int kc = 0; kc < nchunk; ++kc) tma_store_2d(&tmD1, kc * 64, tile * 128, smem_u32(htile + kc * 16384));
-        tma_store_commit_and_wait_read();
-        mbar_arrive(h_empty);
-      }
       ph ^= 1u;
+
+      if (p.fuse && (tile + 1 == t_end || (tile + 1) % tpp == 0)) {
+        // Last tile of partition j in this CTA: deliver [dW2; db2].  Every tensor-core instruction of the tile
+        // has completed (the wait on d_full above).  A partition shared by several CTAs is summed, in CTA
+        // order, by whichever of them delivers last.
+        const int pa = j * tpp, pb = pa + tpp;
+        int cfirst = (int)blockIdx.x, clast = (int)blockIdx.x;
+        while (cfirst > 0 && head_tile_begin(cfirst, p.num_tiles, grid) > pa) --cfirst;
+        while (clast + 1 < grid && head_tile_begin(clast + 1, p.num_tiles, grid) < pb) ++clast;
+        const int nsl = clast - cfirst + 1;
+        float *gdst = p.G + (size_t)j * p.g_batch;
+        float *dst = nsl == 1 ? gdst : p.slots + ((size_t)j * p.max_slots + ((int)blockIdx.x - cfirst)) * wstride;
+        if (part == 0) {
+          for (int mb = 0; mb < p.hidden / 128; ++mb) {
+            float v[16];
+            tmem_ld16(w2_acc + lane_off + (uint32_t)mb * 16u, v);
+            float *o = dst + (size_t)(mb * 128 + r) * p.C;
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              if (c < p.C) o[c] = v[c];
+          }
+          tc_fence_before();
+          if (lane < 16) dbx[q * 16 + lane] = db2_acc;
+          db2_acc = 0.f;
+        }
+        head_epi_sync();
+        if (tid_epi < p.C)
+          dst[(size_t)p.hidden * p.C + tid_epi] = (dbx[tid_epi] + dbx[16 + tid_epi]) + (dbx[32 + tid_epi] + dbx[48 + tid_epi]);
+        if (nsl > 1) {
+          __threadfence();
+          head_epi_sync();
+          if (tid_epi == 0) *last_flag = atomicAdd(p.counters + j, 1) == nsl - 1;
+          head_epi_sync();
+          if (*last_flag) {
+            __threadfence();
+            const float *s0 = p.slots + (size_t)j * p.max_slots * wstride;
+            for (int e = tid_epi; e < wstride; e += kHeadEpiThreads) {
+              float acc = __ldcg(s0 + e);
+              for (int sl = 1; sl < nsl; ++sl) acc += __ldcg(s0 + (size_t)sl * wstride + e);
+              gdst[e] = acc;
+            }
+          }
+        }
+        head_epi_sync();  // last_flag and dbx are free again
+      }
     }
   }
   if (failed) atomicExch(p.status, 1);
@@ -1216,12 +1349,37 @@ namespace {
 inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 }  // namespace
 
+// Largest number of CTAs of the head kernel whose contiguous tile ranges touch one partition.
+static int head_max_slots(int k, int tpp, int grid) {
+  int worst = 1;
+  for (int j = 0; j < k; ++j) {
+    int cnt = 0;
+    for (int c = 0; c < grid; ++c)
+      if (head_tile_begin(c + 1, k * tpp, grid) > j * tpp && head_tile_begin(c, k * tpp, grid) < (j + 1) * tpp) ++cnt;
+    if (cnt > worst) worst = cnt;
+  }
+  return worst;
+}
+
+static int head_grid(int k, int rows, int sms) {
+  const int tiles = k * ((rows + 127) / 128);
+  return tiles < sms ? tiles : (sms > 0 ? sms : 1);
+}
+
 size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
   const size_t dpad = (size_t)(d + 1 + 7) / 8 * 8, hpad = (size_t)(hidden + 1 + 7) / 8 * 8;
   const size_t l = (size_t)d * hidden + hidden + (size_t)hidden * C + C, lpad = (l + 3) / 4 * 4;
   const size_t kr = (size_t)k * rows;
+  const int slots = head_max_slots(k, (rows + 127) / 128, head_grid(k, rows, device_sm_count()));
   return up256(kr * dpad * 2) + up256((size_t)hidden * dpad * 2) + up256(kr * hpad * 2) + up256(kr * hidden * 2) +
-         up256(kr * 64 * 2) + up256((size_t)16 * hidden * 2) + up256((size_t)hidden * 64 * 2) + up256((size_t)k * lpad * 4);
+         up256(kr * 64 * 2) + up256((size_t)16 * hidden * 2) + up256((size_t)hidden * 64 * 2) +
+         up256((size_t)k * slots * ((size_t)hidden * C + C) * 4) + up256((size_t)k * 4) + up256((size_t)k * lpad * 4);
+}
+
+int mlp_launch_count(int hidden) {
+  // convert, transpose, forward, head (+ its operand layouts), dW1, encode; dW2 apart unless the head forms it
+  if (hidden % 128 == 0) return 7;
+  return hidden % 64 == 0 ? 8 : 7;
 }
 
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
@@ -1241,6 +1399,11 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   __nv_bfloat16 *D2 = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256(kr * 64 * 2);
   __nv_bfloat16 *W2t = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)16 * hidden * 2);
   __nv_bfloat16 *W2k = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)hidden * 64 * 2);
+  const int tpp = (rows + 127) / 128, hgrid = head_grid(k, rows, sms);
+  const int max_slots = head_max_slots(k, tpp, head_grid(k, rows, device_sm_count()));
+  if (head_max_slots(k, tpp, hgrid) > max_slots) return cudaErrorInvalidValue;
+  float *slots = reinterpret_cast<float *>(ptr); ptr += up256((size_t)k * max_slots * ((size_t)hidden * C + C) * 4);
+  int *counters = reinterpret_cast<int *>(ptr); ptr += up256((size_t)k * 4);
   float *G = reinterpret_cast<float *>(ptr);
   *G_out = G;
   *G_ld = (long long)lpad;
@@ -1254,8 +1417,9 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   const uint64_t hdims[3] = {(uint64_t)hpad, (uint64_t)rows, (uint64_t)k};
   const uint64_t d1dims[3] = {(uint64_t)hidden, (uint64_t)rows, (uint64_t)k};
   const uint64_t d2dims[3] = {64, (uint64_t)rows, (uint64_t)k};
+  CUtensorMap tmHa;  // h in 128-row boxes (head), tmH in 64-row boxes (backward operand)
   if (!make_map(&tmXa, Xb, 3, xdims, box_a) || !make_map(&tmXb, Xb, 3, xdims, box_b) ||
-      !make_map(&tmW, W1t, 2, wdims, wbox) || !make_map(&tmH, H, 3, hdims, box_b) ||
+      !make_map(&tmW, W1t, 2, wdims, wbox) || !make_map(&tmH, H, 3, hdims, box_b) || !make_map(&tmHa, H, 3, hdims, box_a) ||
       !make_map(&tmD1, D1, 3, d1dims, box_b) || !make_map(&tmD2, D2, 3, d2dims, box_b))
     return cudaErrorInvalidValue;
 
@@ -1276,7 +1440,11 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   FwdParams p;
   p.rows = rows; p.n_total = hidden; p.row_blocks = (rows + 127) / 128; p.n_tiles = (hidden + 255) / 256;
   p.num_tiles = k * p.row_blocks * p.n_tiles; p.num_k = (dpad + 63) / 64;
-  p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = hidden; p.status = status;
+  const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
+  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 512 + 1024;
+  const bool head_tc = hidden % 64 == 0 && head_tc_smem <= 232448;
+  const bool fuse_w2 = head_tc && hidden % 128 == 0;  // the head forms [dW2; db2] itself: no column of ones behind h
+  p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = fuse_w2 ? -1 : hidden; p.status = status;
   const bool pair = (hidden % 256 == 0) && sms >= 2;  // CTA pairs: 256 rows per tile, half of W1^T per CTA
   if (pair) {
     CUtensorMap tmWh;
@@ -1291,25 +1459,25 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   }
   if (e != cudaSuccess) return e;
 
-  const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
-  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 256 + 1024;
-  if (hidden % 64 == 0 && head_tc_smem <= 232448) {
-    CUtensorMap tmH2, tmW2t, tmW2k, tmD1s;
-    const uint64_t h2dims[2] = {(uint64_t)hpad, (uint64_t)kr}, w2tdims[2] = {(uint64_t)hidden, 16},
-                   w2kdims[2] = {64, (uint64_t)hidden}, d1sdims[2] = {(uint64_t)hidden, (uint64_t)kr};
-    const uint32_t box_h[2] = {64, 128}, box_w2t[2] = {64, 16}, box_w2k[2] = {64, 256};
-    if (!make_map(&tmH2, H, 2, h2dims, box_h) || !make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) ||
-        !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) || !make_map(&tmD1s, D1, 2, d1sdims, box_h))
+  if (head_tc) {
+    CUtensorMap tmW2t, tmW2k, tmD1s;
+    const uint64_t w2tdims[2] = {(uint64_t)hidden, 16}, w2kdims[2] = {64, (uint64_t)hidden};
+    const uint32_t box_w2t[2] = {64, 16}, box_w2k[2] = {64, 256};
+    if (!make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) ||
+        !make_map(&tmD1s, D1, 3, d1dims, box_a))
       return cudaErrorInvalidValue;
-    prep_w2_kernel<<<(hidden * 64 + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k);
+    const int prep_n = hidden * 64 > k ? hidden * 64 : k;
+    prep_w2_kernel<<<(prep_n + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k, counters, k);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     HeadTcParams hp;
-    hp.hidden = hidden; hp.C = C; hp.num_tiles = (int)((kr + 127) / 128);
-    hp.b2 = b2; hp.y = y; hp.rows_total = (long long)kr; hp.D2 = D2; hp.status = status;
+    hp.hidden = hidden; hp.C = C; hp.rows = rows; hp.tiles_per_part = tpp; hp.num_tiles = k * tpp;
+    hp.b2 = b2; hp.y = y; hp.D2 = D2; hp.fuse = fuse_w2 ? 1 : 0;
+    hp.slots = slots; hp.max_slots = max_slots; hp.counters = counters;
+    hp.G = G + (size_t)d * hidden + hidden; hp.g_batch = lpad; hp.status = status;
     e = cudaFuncSetAttribute(mlp_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_tc_smem);
     if (e != cudaSuccess) return e;
-    mlp_head_tc_kernel<<<hp.num_tiles < sms ? hp.num_tiles : sms, kHeadTcThreads, head_tc_smem, stream>>>(
-        tmH2, tmW2t, tmW2k, tmD1s, hp);
+    // the same 128 x 64 box serves the loads of h and the stores of delta1
+    mlp_head_tc_kernel<<<hgrid, kHeadTcThreads, head_tc_smem, stream>>>(tmHa, tmW2t, tmW2k, tmD1s, hp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   } else {
     const int cpad = (C + 3) / 4 * 4;
@@ -1344,7 +1512,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmD1, t);
     e = cudaGetLastError();
   }
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || fuse_w2) return e;
   // [dW2; db2] = [h 1]^T delta2
   t.m_tiles = (hidden + 1 + 127) / 128; t.n_tiles = 1; t.num_tiles = k * t.m_tiles;
   t.N = 16; t.nbox = 1;

@@ -56,6 +56,7 @@ cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long
 // MLP (one hidden ReLU layer, softmax cross-entropy) partial gradients on the tensor cores (X fp32):
 // G[k][*G_ld] fp32 inside `scratch`, each row holding [dW1, db1, dW2, db2].
 size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C);
+int mlp_launch_count(int hidden);  // kernels one gradient + encode call launches
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
                             unsigned char *scratch, float **G_out, long long *G_ld, int *status, int sms,
                             cudaStream_t stream);

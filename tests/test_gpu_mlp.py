@@ -25,6 +25,8 @@ CASES = [
     (5, [0, 2], 300, 200, 256, 7, 1),    # ragged rows, odd class count
     (4, [1], 130, 128, 32, 3, 2),        # k = 2 n, narrow hidden layer
     (3, [1], 77, 72, 512, 16, 1),        # widest class count
+    (10, [1], 2000, 64, 128, 10, 1),     # 160 head tiles on 148 CTAs: output-layer sums carried across tiles and CTAs
+    (3, [0], 200, 64, 192, 5, 1),        # hidden not a multiple of 128: output-layer gradient by its own contraction
 ]
 
 
