@@ -527,7 +527,7 @@ mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C
 //      tile's h while the other group is still being worked on.
 // ------------------------------------------------------------------------------------------------
 constexpr int kHeadEpiThreads = 512;  // 16 epilogue warps: four per tensor-memory quadrant
-constexpr int kHeadTcThreads = 64 + kHeadEpiThreads;  // + producer and MMA warps
+constexpr int kHeadTcThreads = 96 + kHeadEpiThreads;  // + two producer warps and the MMA warp
 __device__ __forceinline__ void head_epi_sync() { asm volatile("bar.sync 6, %0;" ::"n"(kHeadEpiThreads) : "memory"); }
 
 struct HeadTcParams {
@@ -538,9 +538,6 @@ struct HeadTcParams {
   int fuse;           // 1: [dW2; db2] = [h 1]^T delta2 is formed here (hidden a multiple of 128)
   float *slots;       // [k][max_slots][hidden * C + C]: partial sums of the CTAs that share a partition
   int max_slots;
-  int *counters;      // [k], zero at launch: CTAs that have delivered their slot of a partition
-  float *G;           // [dW2; db2] of partition j goes to G + j * g_batch
-  size_t g_batch;
   int *status;
 };
 
@@ -548,7 +545,7 @@ struct HeadTcParams {
 __host__ __device__ inline int head_tile_begin(int c, int tiles, int grid) { return (int)((long long)c * tiles / grid); }
 
 __global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, __nv_bfloat16 *__restrict__ W2t,
-                               __nv_bfloat16 *__restrict__ W2k, int *__restrict__ counters, int k) {
+                               __nv_bfloat16 *__restrict__ W2k) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < 16 * hidden) {  // W2t[c][hc]
     const int c = i / hidden, hc = i % hidden;
@@ -558,7 +555,6 @@ __global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, 
     const int hc = i / 64, c = i % 64;
     W2k[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
   }
-  if (i < k) counters[i] = 0;
 }
 
 __global__ void __launch_bounds__(kHeadTcThreads, 1)
@@ -577,18 +573,18 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   // The tile lives in shared memory as groups of two 64-column chunks.  Group g is loaded (h), consumed,
   // overwritten in place (delta1), stored and reloaded with the next tile's h on its own barriers, so the
   // memory traffic of the finished groups hides behind the arithmetic on the others.
-  uint32_t h_full[4], m_done[4];
+  uint32_t h_full[4], m_done[4], w_done[4];
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     h_full[g] = smem_u32(&bars[g]);
     m_done[g] = smem_u32(&bars[4 + g]);
+    w_done[g] = smem_u32(&bars[8 + g]);
   }
-  const uint32_t z_full = smem_u32(&bars[8]), d2_full = smem_u32(&bars[9]), d_full = smem_u32(&bars[10]),
-                 d_empty = smem_u32(&bars[11]), w_full = smem_u32(&bars[12]);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[13]);
-  float *b2s = reinterpret_cast<float *>(&bars[14]);          // 16 floats
-  float *dbx = reinterpret_cast<float *>(&bars[22]);          // [4 quadrants][16]: bias-gradient partial sums
-  volatile int *last_flag = reinterpret_cast<volatile int *>(&bars[54]);
+  const uint32_t z_full = smem_u32(&bars[12]), d2_full = smem_u32(&bars[13]), d_full = smem_u32(&bars[14]),
+                 d_empty = smem_u32(&bars[15]), w_full = smem_u32(&bars[16]);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[17]);
+  float *b2s = reinterpret_cast<float *>(&bars[18]);          // 16 floats
+  float *dbx = reinterpret_cast<float *>(&bars[26]);          // [4 quadrants][16]: bias-gradient partial sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -596,6 +592,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
     for (int g = 0; g < 4; ++g) {
       mbar_init(h_full[g], 1);
       mbar_init(m_done[g], kHeadEpiThreads);
+      mbar_init(w_done[g], 1);
     }
     mbar_init(z_full, 1);
     mbar_init(d2_full, 128);
@@ -616,22 +613,27 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   const int t_begin = head_tile_begin((int)blockIdx.x, p.num_tiles, grid),
             t_end = head_tile_begin((int)blockIdx.x + 1, p.num_tiles, grid);
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 2) {
+    // Two producers: warp 0 owns the even chunk groups, warp 2 the odd ones, so that one of them can wait for
+    // a store to release its group while the other already handles the next group.
     if (lane == 0) {
-      mbar_expect_tx(w_full, (uint32_t)(nchunk * 2048 + nhalf * 32768));
-      for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(w2t + kc * 2048), &tmW2t, kc * 64, 0, w_full);
-      for (int hh = 0; hh < nhalf; ++hh) tma_load_2d(smem_u32(w2k + hh * 32768), &tmW2k, 0, hh * 256, w_full);
+      const int g0 = warp >> 1;
+      if (warp == 0) {
+        mbar_expect_tx(w_full, (uint32_t)(nchunk * 2048 + nhalf * 32768));
+        for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(w2t + kc * 2048), &tmW2t, kc * 64, 0, w_full);
+        for (int hh = 0; hh < nhalf; ++hh) tma_load_2d(smem_u32(w2k + hh * 32768), &tmW2k, 0, hh * 256, w_full);
+      }
       auto load_group = [&](int tile, int g) {
         const int j = tile / tpp, rb = tile % tpp, c0 = g * 2, c1 = min(nchunk, c0 + 2);
         mbar_expect_tx(h_full[g], (uint32_t)(c1 - c0) * 16384u);
         for (int kc = c0; kc < c1; ++kc)
           tma_load_3d(smem_u32(htile + kc * 16384), &tmH, kc * 64, rb * 128, j, h_full[g]);
       };
-      for (int g = 0; g < ngroups; ++g) load_group(t_begin, g);
+      for (int g = g0; g < ngroups; g += 2) load_group(t_begin, g);
       uint32_t ph = 0;
       for (int tile = t_begin; tile < t_end && !failed; ++tile) {
         const int j = tile / tpp, rb = tile % tpp;
-        for (int g = 0; g < ngroups; ++g) {
+        for (int g = g0; g < ngroups; g += 2) {
           // delta1 has replaced h in group g: store it, and once the store has read shared memory bring the
           // next tile's h into the same chunks
           if (!mbar_wait(m_done[g], ph)) { failed = true; break; }
@@ -669,19 +671,6 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
         const uint64_t ad1 = smem_desc_sw128(smem_u32(d2tile), 16, 1024);      // delta2, K-major (K = classes)
         const uint64_t bdw = smem_desc_sw128(smem_u32(d2tile), 16384, 1024);   // delta2, N-major (K = samples)
         for (int hh = 0; hh < nhalf; ++hh) {
-          if (p.fuse) {
-            // dW2 block (128 hidden units x 16 classes) += h_block^T delta2 for the blocks inside this half:
-            // both operands are read M/N-major from the tiles the other contractions use K-major.  Issued
-            // ahead of the half's delta1 contraction, whose commit therefore covers them too: h may be
-            // overwritten once d_full has fired.  The second half's share runs under the first mask pass.
-            for (int mb = hh * 2; mb < min(nmb, hh * 2 + 2); ++mb) {
-              const uint64_t adw = smem_desc_sw128(smem_u32(htile + mb * 32768), 16384, 1024);
-#pragma unroll
-              for (int k8 = 0; k8 < 8; ++k8)  // 16 samples = 2048 bytes per instruction
-                mma_bf16(w2_acc + (uint32_t)mb * 16u, adw + (uint64_t)(k8 * 128), bdw + (uint64_t)(k8 * 128), idesc_w,
-                         !(first && k8 == 0));
-            }
-          }
           if (!mbar_wait(d_empty, dph ^ 1u)) { failed = true; break; }
           tc_fence_after();
           const int nh = min(256, p.hidden - hh * 256);
@@ -689,14 +678,28 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
           mma_bf16(d_acc, ad1, bd, instr_desc_bf16(128, nh, 0, 0), 0);  // K = 16: the 16 class columns
           mma_commit(d_full);
           dph ^= 1u;
+          if (p.fuse) {
+            // dW2 block (128 hidden units x 16 classes) += h_block^T delta2 for the two blocks inside this half:
+            // both operands are read M/N-major from the tiles the other contractions use K-major.  They run
+            // while the epilogue fetches the delta1 accumulator; block mb = chunk group mb may be overwritten
+            // once w_done[mb] has fired.
+            for (int mb = hh * 2; mb < min(nmb, hh * 2 + 2); ++mb) {
+              const uint64_t adw = smem_desc_sw128(smem_u32(htile + mb * 32768), 16384, 1024);
+#pragma unroll
+              for (int k8 = 0; k8 < 8; ++k8)  // 16 samples = 2048 bytes per instruction
+                mma_bf16(w2_acc + (uint32_t)mb * 16u, adw + (uint64_t)(k8 * 128), bdw + (uint64_t)(k8 * 128), idesc_w,
+                         !(first && k8 == 0));
+              mma_commit(w_done[mb]);
+            }
+          }
         }
         ph ^= 1u;
       }
     }
   } else {
     const int q = warp & 3, r = q * 32 + lane;  // row of the tile = tensor-memory lane
-    const int part = (warp - 2) >> 2;           // the four warps of a quadrant split every chunk: 16 columns each
-    const int tid_epi = (int)threadIdx.x - 64;
+    const int part = (warp - 3) >> 2;           // the four warps of a quadrant split every chunk: 16 columns each
+    const int tid_epi = (int)threadIdx.x - 96;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;  // row r inside a swizzled tile
     const uint32_t rx = (uint32_t)(r & 7);
@@ -774,6 +777,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
           mbar_arrive(d_empty);
           dph ^= 1u;
         }
+        if (p.fuse && !mbar_wait(w_done[g], ph)) { failed = true; break; }  // the tensor cores are done with h
         const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
@@ -808,16 +812,12 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       ph ^= 1u;
 
       if (p.fuse && (tile + 1 == t_end || (tile + 1) % tpp == 0)) {
-        // Last tile of partition j in this CTA: deliver [dW2; db2].  Every tensor-core instruction of the tile
-        // has completed (the wait on d_full above).  A partition shared by several CTAs is summed, in CTA
-        // order, by whichever of them delivers last.
-        const int pa = j * tpp, pb = pa + tpp;
-        int cfirst = (int)blockIdx.x, clast = (int)blockIdx.x;
-        while (cfirst > 0 && head_tile_begin(cfirst, p.num_tiles, grid) > pa) --cfirst;
-        while (clast + 1 < grid && head_tile_begin(clast + 1, p.num_tiles, grid) < pb) ++clast;
-        const int nsl = clast - cfirst + 1;
-        float *gdst = p.G + (size_t)j * p.g_batch;
-        float *dst = nsl == 1 ? gdst : p.slots + ((size_t)j * p.max_slots + ((int)blockIdx.x - cfirst)) * wstride;
+        // Last tile of partition j in this CTA: deliver this CTA's share of [dW2; db2] to its slot.  Every
+        // tensor-core instruction of the tile has completed (the wait on w_done of the last group above).
+        // `head_reduce_kernel` adds up the slots of a partition in CTA order.
+        int cfirst = (int)blockIdx.x;
+        while (cfirst > 0 && head_tile_begin(cfirst, p.num_tiles, grid) > j * tpp) --cfirst;
+        float *dst = p.slots + ((size_t)j * p.max_slots + ((int)blockIdx.x - cfirst)) * wstride;
         if (part == 0) {
           for (int mb = 0; mb < p.hidden / 128; ++mb) {
             float v[16];
@@ -834,22 +834,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
         head_epi_sync();
         if (tid_epi < p.C)
           dst[(size_t)p.hidden * p.C + tid_epi] = (dbx[tid_epi] + dbx[16 + tid_epi]) + (dbx[32 + tid_epi] + dbx[48 + tid_epi]);
-        if (nsl > 1) {
-          __threadfence();
-          head_epi_sync();
-          if (tid_epi == 0) *last_flag = atomicAdd(p.counters + j, 1) == nsl - 1;
-          head_epi_sync();
-          if (*last_flag) {
-            __threadfence();
-            const float *s0 = p.slots + (size_t)j * p.max_slots * wstride;
-            for (int e = tid_epi; e < wstride; e += kHeadEpiThreads) {
-              float acc = __ldcg(s0 + e);
-              for (int sl = 1; sl < nsl; ++sl) acc += __ldcg(s0 + (size_t)sl * wstride + e);
-              gdst[e] = acc;
-            }
-          }
-        }
-        head_epi_sync();  // last_flag and dbx are free again
+        head_epi_sync();  // dbx is free again
       }
     }
   }
@@ -857,6 +842,21 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// [dW2; db2] of partition j = sum of the slots the head kernel's CTAs filled, in CTA order (reruns are
+// bit-identical).  blockIdx.y = partition.
+__global__ void head_reduce_kernel(const float *__restrict__ slots, int max_slots, int wstride, int tpp, int num_tiles,
+                                   int grid, float *__restrict__ G, size_t g_batch) {
+  const int j = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= wstride) return;
+  // CTAs of the head kernel whose tile range meets partition j
+  const int cfirst = (int)(((long long)(j * tpp + 1) * grid - 1) / num_tiles);
+  const int clast = (int)(((long long)((j + 1) * tpp) * grid - 1) / num_tiles);
+  const float *s0 = slots + (size_t)j * max_slots * wstride + e;
+  float acc = s0[0];
+  for (int sl = 1; sl <= clast - cfirst; ++sl) acc += s0[(size_t)sl * wstride];
+  G[(size_t)j * g_batch + e] = acc;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1373,12 +1373,12 @@ size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
   const int slots = head_max_slots(k, (rows + 127) / 128, head_grid(k, rows, device_sm_count()));
   return up256(kr * dpad * 2) + up256((size_t)hidden * dpad * 2) + up256(kr * hpad * 2) + up256(kr * hidden * 2) +
          up256(kr * 64 * 2) + up256((size_t)16 * hidden * 2) + up256((size_t)hidden * 64 * 2) +
-         up256((size_t)k * slots * ((size_t)hidden * C + C) * 4) + up256((size_t)k * 4) + up256((size_t)k * lpad * 4);
+         up256((size_t)k * slots * ((size_t)hidden * C + C) * 4) + up256((size_t)k * lpad * 4);
 }
 
 int mlp_launch_count(int hidden) {
-  // convert, transpose, forward, head (+ its operand layouts), dW1, encode; dW2 apart unless the head forms it
-  if (hidden % 128 == 0) return 7;
+  // convert, transpose, forward, head (+ its operand layouts), dW1, encode; dW2 by a contraction of its own, or
+  // by the head kernel plus the sum over its slots
   return hidden % 64 == 0 ? 8 : 7;
 }
 
@@ -1403,7 +1403,6 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   const int max_slots = head_max_slots(k, tpp, head_grid(k, rows, device_sm_count()));
   if (head_max_slots(k, tpp, hgrid) > max_slots) return cudaErrorInvalidValue;
   float *slots = reinterpret_cast<float *>(ptr); ptr += up256((size_t)k * max_slots * ((size_t)hidden * C + C) * 4);
-  int *counters = reinterpret_cast<int *>(ptr); ptr += up256((size_t)k * 4);
   float *G = reinterpret_cast<float *>(ptr);
   *G_out = G;
   *G_ld = (long long)lpad;
@@ -1466,19 +1465,23 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     if (!make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) ||
         !make_map(&tmD1s, D1, 3, d1dims, box_a))
       return cudaErrorInvalidValue;
-    const int prep_n = hidden * 64 > k ? hidden * 64 : k;
-    prep_w2_kernel<<<(prep_n + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k, counters, k);
+    prep_w2_kernel<<<(hidden * 64 + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     HeadTcParams hp;
     hp.hidden = hidden; hp.C = C; hp.rows = rows; hp.tiles_per_part = tpp; hp.num_tiles = k * tpp;
     hp.b2 = b2; hp.y = y; hp.D2 = D2; hp.fuse = fuse_w2 ? 1 : 0;
-    hp.slots = slots; hp.max_slots = max_slots; hp.counters = counters;
-    hp.G = G + (size_t)d * hidden + hidden; hp.g_batch = lpad; hp.status = status;
+    hp.slots = slots; hp.max_slots = max_slots; hp.status = status;
     e = cudaFuncSetAttribute(mlp_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_tc_smem);
     if (e != cudaSuccess) return e;
     // the same 128 x 64 box serves the loads of h and the stores of delta1
     mlp_head_tc_kernel<<<hgrid, kHeadTcThreads, head_tc_smem, stream>>>(tmHa, tmW2t, tmW2k, tmD1s, hp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (fuse_w2) {
+      const int wstride = hidden * C + C;
+      head_reduce_kernel<<<dim3((wstride + 255) / 256, k), 256, 0, stream>>>(slots, max_slots, wstride, tpp, k * tpp, hgrid,
+                                                                            G + (size_t)d * hidden + hidden, lpad);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
   } else {
     const int cpad = (C + 3) / 4 * 4;
     const size_t head_smem = ((size_t)hidden * cpad + cpad + 4 * kHeadRows * cpad) * sizeof(float) + (size_t)kHeadRows * hpad * 2;
