@@ -1207,18 +1207,180 @@ tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   pair_teardown(warp, tmem_base, failed, p.status);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Wide backward contraction on a CTA pair, roles swapped: D^T = A^T B with A [batch][K][M] on the M side in
+// blocks of 256 (128 per CTA) and B [batch][K][n_total] on the N side in passes of up to 512 columns, so that
+// one pass fills all of tensor memory (two accumulators of up to 256 columns) and the A block is fetched once
+// per 512 columns of B instead of once per 256.  These kernels run at the rate shared memory is fed from L2,
+// not at the tensor cores' rate: a pass moves 96 KB per K chunk for 256 x 512 outputs where two 256 x 256
+// tiles move 128 KB.  A ragged last pass issues a narrower second instruction (N a multiple of 32) instead of
+// a whole padded tile.  D^T(m, n) is stored at out[n * out_ld + m]: consecutive lanes hold consecutive m, so
+// every column of the accumulator leaves as one 128-byte warp store.
+// Unit = (batch j, M block mt, pass p), mt fastest (neighbouring pairs share B through L2), batches last to
+// first (the kernel before went first to last).  Units go round-robin to the pairs.
+// ------------------------------------------------------------------------------------------------
+constexpr int kWideStages = 4;
+constexpr int kWideStageBytes = 16384 + 4 * 8192;  // 128 x 64 of A + up to four 64 x 64 boxes of B per CTA
+constexpr int kSmemWide = kWideStages * kWideStageBytes + 1024 + 256;
+constexpr int kWideThreads = 320;  // producer, MMA, 8 epilogue warps
+
+struct TnWideParams {
+  int batch, m_tiles, n_passes, num_units;
+  int num_k;      // K chunks of 64
+  int n_total;    // columns of B that exist in D^T (rows of the stored matrix)
+  float *out;     // D^T(j, m, n) -> out[j * out_batch + n * out_ld + m]
+  size_t out_batch;
+  int out_ld;
+  int *status;
+};
+
+// Widths of the two instructions of pass `pass` (multiples of 32; w1 may be 0).
+__host__ __device__ inline void wide_pass_widths(int n_total, int pass, int *w0, int *w1) {
+  const int rem = n_total - pass * 512;
+  const int r32 = (rem + 31) / 32 * 32;
+  *w0 = r32 < 256 ? r32 : 256;
+  const int r1 = r32 - 256;
+  *w1 = r1 <= 0 ? 0 : (r1 < 256 ? r1 : 256);
+}
+
+__global__ void __launch_bounds__(kWideThreads, 1)
+tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const TnWideParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t sbase = smem_u32(smem_raw);
+  unsigned char *tiles = smem_raw + ((1024u - (sbase & 1023u)) & 1023u);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + kWideStages * kWideStageBytes);
+  uint32_t full[kWideStages], empty[kWideStages];
+#pragma unroll
+  for (int i = 0; i < kWideStages; ++i) {
+    full[i] = smem_u32(&bars[i]);
+    empty[i] = smem_u32(&bars[kWideStages + i]);
+  }
+  const uint32_t tfull = smem_u32(&bars[2 * kWideStages]), tempty = smem_u32(&bars[2 * kWideStages + 1]);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kWideStages + 2]);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kWideStages; ++i) {
+      mbar_init(full[i], 1);
+      mbar_init(empty[i], 1);
+    }
+    mbar_init(tfull, 1);
+    mbar_init(tempty, 2 * (kWideThreads - 64));
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  bool failed = false;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int per_batch = p.m_tiles * p.n_passes;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int st = 0;
+      uint32_t ph = 0;
+      for (int u = pair_id; u < p.num_units && !failed; u += n_pairs) {
+        const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
+        int w0, w1;
+        wide_pass_widths(p.n_total, pass, &w0, &w1);
+        const int nb0 = (w0 / 2 + 63) / 64, nb1 = (w1 / 2 + 63) / 64;  // 64-column boxes of B this CTA loads
+        const int m0 = mt * 256 + (int)rank * 128;
+        const int c0 = pass * 512 + (int)rank * (w0 / 2), c1 = pass * 512 + 256 + (int)rank * (w1 / 2);
+        const uint32_t tx = 2u * (16384u + (uint32_t)(nb0 + nb1) * 8192u);  // both CTAs signal the leader's barrier
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(empty[st], ph ^ 1u)) { failed = true; break; }
+          if (rank == 0) mbar_expect_tx(full[st], tx);
+          const uint32_t a = smem_u32(tiles + st * kWideStageBytes);
+          const uint32_t bar = map_to_rank(full[st], 0);
+          tma_load_3d_pair(a, &tmA, m0, kc * 64, j, bar);
+          tma_load_3d_pair(a + 8192, &tmA, m0 + 64, kc * 64, j, bar);
+          for (int b = 0; b < nb0; ++b) tma_load_3d_pair(a + 16384 + b * 8192, &tmB, c0 + b * 64, kc * 64, j, bar);
+          for (int b = 0; b < nb1; ++b)
+            tma_load_3d_pair(a + 16384 + (nb0 + b) * 8192, &tmB, c1 + b * 64, kc * 64, j, bar);
+          if (++st == kWideStages) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      int st = 0;
+      uint32_t ph = 0, aph = 0;
+      for (int u = pair_id; u < p.num_units && !failed; u += n_pairs) {
+        const int pass = (u % per_batch) / p.m_tiles;
+        int w0, w1;
+        wide_pass_widths(p.n_total, pass, &w0, &w1);
+        const int nb0 = (w0 / 2 + 63) / 64;
+        const uint32_t idesc0 = instr_desc_bf16(256, w0, 1, 1), idesc1 = instr_desc_bf16(256, w1 ? w1 : 32, 1, 1);
+        if (!mbar_wait(tempty, aph ^ 1u)) { failed = true; break; }
+        tc_fence_after();
+        for (int kc = 0; kc < p.num_k; ++kc) {
+          if (!mbar_wait(full[st], ph)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a = smem_u32(tiles + st * kWideStageBytes);
+          // M/N-major: 64-element boxes 8192 B apart, 8-row K groups 1024 B apart
+          const uint64_t ad = smem_desc_sw128(a, 8192, 1024), bd0 = smem_desc_sw128(a + 16384, 8192, 1024),
+                         bd1 = smem_desc_sw128(a + 16384 + nb0 * 8192, 8192, 1024);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) {  // 16 rows of K = 2048 bytes per instruction
+            mma_bf16_pair(tmem_base, ad + (uint64_t)(k4 * 128), bd0 + (uint64_t)(k4 * 128), idesc0, (kc | k4) != 0);
+            if (w1)
+              mma_bf16_pair(tmem_base + 256u, ad + (uint64_t)(k4 * 128), bd1 + (uint64_t)(k4 * 128), idesc1, (kc | k4) != 0);
+          }
+          mma_commit_pair(empty[st], 3);
+          if (++st == kWideStages) { st = 0; ph ^= 1u; }
+        }
+        if (failed) break;
+        mma_commit_pair(tfull, 3);
+        aph ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3, half = (warp - 2) >> 2;  // warps w and w + 4 share a quadrant and alternate 32-column chunks
+    uint32_t aph = 0;
+    for (int u = pair_id; u < p.num_units; u += n_pairs) {
+      const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
+      int w0, w1;
+      wide_pass_widths(p.n_total, pass, &w0, &w1);
+      if (!mbar_wait(tfull, aph)) { failed = true; break; }
+      tc_fence_after();
+      const int m = mt * 256 + (int)rank * 128 + q * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      float *dst = p.out + (size_t)j * p.out_batch + m;
+      const int ch0 = w0 >> 5, chunks = ch0 + (w1 >> 5);
+      for (int ch = half; ch < chunks; ch += 2) {
+        const int col = ch < ch0 ? ch * 32 : 256 + (ch - ch0) * 32;  // accumulator column = column of the pass
+        const int n0 = pass * 512 + col;
+        if (n0 >= p.n_total) continue;  // (uniform per warp)
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)col, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (n0 + i < p.n_total) dst[(size_t)(n0 + i) * p.out_ld] = v[i];
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_rank(tempty, 0));
+      aph ^= 1u;
+    }
+  }
+  pair_teardown(warp, tmem_base, failed, p.status);
+}
+
 // Launch on clusters of two CTAs.
 template <typename Kern, typename Params>
 cudaError_t launch_pair(Kern kern, int threads, int pair_tiles, int sms, const CUtensorMap &m0, const CUtensorMap &m1,
-                        const Params &p, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPair);
+                        const Params &p, cudaStream_t stream, int smem_bytes = kSmemPair) {
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   int pairs = sms / 2;
   if (pair_tiles < pairs) pairs = pair_tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(threads);
-  cfg.dynamicSmemBytes = kSmemPair;
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1509,8 +1671,12 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   t.m_store = d + 1; t.n_store = t.N;
   t.out = G; t.out_batch = lpad; t.out_ld = hidden;
   if (pair) {
-    t.m_tiles = (d + 1 + 255) / 256; t.num_tiles = k * t.m_tiles * t.n_tiles;
-    e = launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, tmXb, tmD1, t, stream);
+    // delta1 on the M side (hidden is a multiple of 256), [X 1] on the N side in passes of 512 columns
+    TnWideParams wp;
+    wp.batch = k; wp.m_tiles = hidden / 256; wp.n_passes = (d + 1 + 511) / 512;
+    wp.num_units = k * wp.m_tiles * wp.n_passes; wp.num_k = (rows + 63) / 64;
+    wp.n_total = d + 1; wp.out = G; wp.out_batch = lpad; wp.out_ld = hidden; wp.status = status;
+    e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, tmD1, tmXb, wp, stream, kSmemWide);
   } else {
     tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmD1, t);
     e = cudaGetLastError();
