@@ -134,33 +134,42 @@ __device__ __forceinline__ void epilogue_teardown(const Smem &s, int warp, uint3
 // bias vector, column d of W^T holds it (the data matrix then carries a matching column of ones);
 // columns beyond are zero.
 // ------------------------------------------------------------------------------------------------
-__global__ void transpose_to_bf16_kernel(const float *__restrict__ W, const float *__restrict__ bias,
-                                         __nv_bfloat16 *__restrict__ Wt, int d, int C, int ld) {
-  __shared__ float tile[32][33];
-  const int c0 = blockIdx.x * 32, d0 = blockIdx.y * 32;
-  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
-    const int dd = d0 + r, c = c0 + threadIdx.x;
+// One 32 x 32 tile (bx along C, by along d) by a block of 256 threads.
+__device__ __forceinline__ void transpose_tile_to_bf16(const float *__restrict__ W, const float *__restrict__ bias,
+                                                       __nv_bfloat16 *__restrict__ Wt, int d, int C, int ld, int bx,
+                                                       int by, float (*tile)[33]) {
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int c0 = bx * 32, d0 = by * 32;
+  for (int r = ty; r < 32; r += 8) {
+    const int dd = d0 + r, c = c0 + tx;
     float v = 0.f;
     if (c < C) {
       if (dd < d) v = W[(size_t)dd * C + c];
       else if (dd == d && bias) v = bias[c];
     }
-    tile[r][threadIdx.x] = v;
+    tile[r][tx] = v;
   }
   __syncthreads();
-  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
-    const int c = c0 + r, dd = d0 + threadIdx.x;
-    if (c < C && dd < ld) Wt[(size_t)c * ld + dd] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+  for (int r = ty; r < 32; r += 8) {
+    const int c = c0 + r, dd = d0 + tx;
+    if (c < C && dd < ld) Wt[(size_t)c * ld + dd] = __float2bfloat16_rn(tile[tx][r]);
   }
+}
+
+__global__ void __launch_bounds__(256)
+transpose_to_bf16_kernel(const float *__restrict__ W, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ Wt,
+                         int d, int C, int ld) {
+  __shared__ float tile[32][33];
+  transpose_tile_to_bf16(W, bias, Wt, d, C, ld, blockIdx.x, blockIdx.y, tile);
 }
 
 // X (fp32, [rows_total][d]) -> bf16 [rows_total][ld] with a column of ones at index d and zeros after
 // it: the ones column turns the bias of the first layer, and the bias gradient, into one more row of
 // the weight contraction.  One thread per 8 output columns.
-__global__ void convert_x_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ Xb, long long rows_total,
-                                 int d, int ld) {
+__device__ __forceinline__ void convert_x_block(const float *__restrict__ X, __nv_bfloat16 *__restrict__ Xb,
+                                                long long rows_total, int d, int ld, long long block) {
   const int groups = ld / 8;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long idx = block * blockDim.x + threadIdx.x;
   if (idx >= rows_total * groups) return;
   const long long row = idx / groups;
   const int c0 = (int)(idx % groups) * 8;
@@ -544,9 +553,9 @@ struct HeadTcParams {
 // Tiles [begin, end) of CTA c when `tiles` tiles are cut into `grid` contiguous ranges.
 __host__ __device__ inline int head_tile_begin(int c, int tiles, int grid) { return (int)((long long)c * tiles / grid); }
 
-__global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, __nv_bfloat16 *__restrict__ W2t,
-                               __nv_bfloat16 *__restrict__ W2k) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void prep_w2_block(const float *__restrict__ W2, int hidden, int C,
+                                              __nv_bfloat16 *__restrict__ W2t, __nv_bfloat16 *__restrict__ W2k, int block) {
+  const int i = block * blockDim.x + threadIdx.x;
   if (i < 16 * hidden) {  // W2t[c][hc]
     const int c = i / hidden, hc = i % hidden;
     W2t[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
@@ -555,6 +564,33 @@ __global__ void prep_w2_kernel(const float *__restrict__ W2, int hidden, int C, 
     const int hc = i / 64, c = i % 64;
     W2k[i] = __float2bfloat16_rn(c < C ? W2[(size_t)hc * C + c] : 0.f);
   }
+}
+
+// Everything the MLP gradient needs before its first contraction, in one launch of 256-thread blocks: the
+// data matrix as bf16 with a column of ones (the bulk of the blocks, bound by HBM), W1 / b1 transposed to the
+// K-major operand of the forward contraction, and (w2_blocks > 0) the two layouts of W2 the head reads.  The
+// small jobs sit at the front of the grid and finish under the conversion.
+struct MlpPrepParams {
+  const float *X; __nv_bfloat16 *Xb; long long rows_total; int d, dpad;
+  const float *W1, *b1; __nv_bfloat16 *W1t; int hidden;
+  const float *W2; int C; __nv_bfloat16 *W2t, *W2k;
+  int tr_bx, tr_blocks, w2_blocks;
+};
+
+__global__ void __launch_bounds__(256) mlp_prep_kernel(const MlpPrepParams p) {
+  __shared__ float tile[32][33];
+  int b = blockIdx.x;
+  if (b < p.tr_blocks) {
+    transpose_tile_to_bf16(p.W1, p.b1, p.W1t, p.d, p.hidden, p.dpad, b % p.tr_bx, b / p.tr_bx, tile);
+    return;
+  }
+  b -= p.tr_blocks;
+  if (b < p.w2_blocks) {
+    prep_w2_block(p.W2, p.hidden, p.C, p.W2t, p.W2k, b);
+    return;
+  }
+  b -= p.w2_blocks;
+  convert_x_block(p.X, p.Xb, p.rows_total, p.d, p.dpad, b);
 }
 
 __global__ void __launch_bounds__(kHeadTcThreads, 1)
@@ -1461,8 +1497,8 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
       !make_map(&tmW, Wt, 2, wdims, wbox) || !make_map(&tmR, R, 3, rdims, rbox))
     return cudaErrorInvalidValue;
 
-  dim3 tb(32, 8), tg((C + 31) / 32, (d + 31) / 32);
-  transpose_to_bf16_kernel<<<tg, tb, 0, stream>>>(W, nullptr, Wt, d, C, d);
+  dim3 tg((C + 31) / 32, (d + 31) / 32);
+  transpose_to_bf16_kernel<<<tg, 256, 0, stream>>>(W, nullptr, Wt, d, C, d);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
@@ -1539,9 +1575,10 @@ size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
 }
 
 int mlp_launch_count(int hidden) {
-  // convert, transpose, forward, head (+ its operand layouts), dW1, encode; dW2 by a contraction of its own, or
-  // by the head kernel plus the sum over its slots
-  return hidden % 64 == 0 ? 8 : 7;
+  // operand preparation, forward, head, dW1, encode; dW2 by a contraction of its own, or by the head kernel
+  // plus the sum over its slots
+  (void)hidden;
+  return 6;
 }
 
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
@@ -1584,13 +1621,21 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
       !make_map(&tmD1, D1, 3, d1dims, box_b) || !make_map(&tmD2, D2, 3, d2dims, box_b))
     return cudaErrorInvalidValue;
 
+  const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
+  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 512 + 1024;
+  const bool head_tc = hidden % 64 == 0 && head_tc_smem <= 232448;
+  const bool fuse_w2 = head_tc && hidden % 128 == 0;  // the head forms [dW2; db2] itself: no column of ones behind h
+
+  MlpPrepParams pp;
+  pp.X = X; pp.Xb = Xb; pp.rows_total = (long long)kr; pp.d = d; pp.dpad = dpad;
+  pp.W1 = W1; pp.b1 = b1; pp.W1t = W1t; pp.hidden = hidden;
+  pp.W2 = W2; pp.C = C; pp.W2t = W2t; pp.W2k = W2k;
+  pp.tr_bx = (hidden + 31) / 32; pp.tr_blocks = pp.tr_bx * ((dpad + 31) / 32);
+  pp.w2_blocks = head_tc ? (hidden * 64 + 255) / 256 : 0;
   const long long groups = (long long)kr * (dpad / 8);
-  convert_x_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, stream>>>(X, Xb, (long long)kr, d, dpad);
+  mlp_prep_kernel<<<(unsigned)(pp.tr_blocks + pp.w2_blocks + (groups + 255) / 256), 256, 0, stream>>>(pp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  dim3 tb(32, 8), tg((hidden + 31) / 32, (dpad + 31) / 32);
-  transpose_to_bf16_kernel<<<tg, tb, 0, stream>>>(W1, b1, W1t, d, hidden, dpad);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   e = cudaFuncSetAttribute(fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFwd);
   if (e != cudaSuccess) return e;
@@ -1601,10 +1646,6 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   FwdParams p;
   p.rows = rows; p.n_total = hidden; p.row_blocks = (rows + 127) / 128; p.n_tiles = (hidden + 255) / 256;
   p.num_tiles = k * p.row_blocks * p.n_tiles; p.num_k = (dpad + 63) / 64;
-  const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
-  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 512 + 1024;
-  const bool head_tc = hidden % 64 == 0 && head_tc_smem <= 232448;
-  const bool fuse_w2 = head_tc && hidden % 128 == 0;  // the head forms [dW2; db2] itself: no column of ones behind h
   p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = fuse_w2 ? -1 : hidden; p.status = status;
   const bool pair = (hidden % 256 == 0) && sms >= 2;  // CTA pairs: 256 rows per tile, half of W1^T per CTA
   if (pair) {
@@ -1627,8 +1668,6 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     if (!make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) ||
         !make_map(&tmD1s, D1, 3, d1dims, box_a))
       return cudaErrorInvalidValue;
-    prep_w2_kernel<<<(hidden * 64 + 255) / 256, 256, 0, stream>>>(W2, hidden, C, W2t, W2k);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     HeadTcParams hp;
     hp.hidden = hidden; hp.C = C; hp.rows = rows; hp.tiles_per_part = tpp; hp.num_tiles = k * tpp;
     hp.b2 = b2; hp.y = y; hp.D2 = D2; hp.fuse = fuse_w2 ? 1 : 0;
