@@ -890,8 +890,15 @@ __global__ void head_reduce_kernel(const float *__restrict__ slots, int max_slot
   const int cfirst = (int)(((long long)(j * tpp + 1) * grid - 1) / num_tiles);
   const int clast = (int)(((long long)((j + 1) * tpp) * grid - 1) / num_tiles);
   const float *s0 = slots + (size_t)j * max_slots * wstride + e;
-  float acc = s0[0];
-  for (int sl = 1; sl <= clast - cfirst; ++sl) acc += s0[(size_t)sl * wstride];
+  const int nsl = clast - cfirst + 1;
+  float acc = 0.f;
+  for (int sb = 0; sb < nsl; sb += 8) {  // eight loads in flight, added in slot order
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = sb + i < nsl ? __ldg(s0 + (size_t)(sb + i) * wstride) : 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc += v[i];
+  }
   G[(size_t)j * g_batch + e] = acc;
 }
 
