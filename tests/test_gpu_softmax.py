@@ -25,6 +25,9 @@ CASES = [
     (5, [0, 2], 300, 192, 80, 1),      # ragged rows (300 = 2*128+44), ragged feature block, C not a multiple of 64
     (6, [1, 3], 1000, 512, 128, 1),
     (4, [1], 130, 128, 16, 2),         # k = 2 n, smallest class count
+    (4, [1], 520, 1032, 256, 1),       # CTA-pair kernels: ragged 256-row blocks, five feature blocks (the last 8 wide)
+    (2, [1], 200, 128, 256, 2),        # k = 2 n with full-width classes, less than one 256-row block
+    (2, [0], 256, 64, 256, 2),         # ... exactly one block, a single K chunk in the forward pass
 ]
 
 
