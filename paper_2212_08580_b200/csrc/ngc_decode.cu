@@ -4,6 +4,7 @@
 //   * the decode itself, g = sum_{i in S} a_i x_i (Section II-C), a bandwidth-bound weighted
 //     reduction over the coded gradients.
 #include "ngc_device.h"
+#include "ngc_pdl.cuh"
 
 namespace ngc {
 
@@ -30,6 +31,7 @@ __global__ void __launch_bounds__(kSolveWarps * 32)
 decode_solve_kernel(const uint64_t *__restrict__ masks, MaskArg one, int batch, int n, int s,
                     const double *__restrict__ a0, const double *__restrict__ Nmat, const double *__restrict__ coef,
                     double *__restrict__ a_out, double *__restrict__ resid_out, double *maxres) {
+  pdl_sync();
   extern __shared__ __align__(16) unsigned char solve_smem[];
   const int warps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -133,6 +135,7 @@ constexpr int kDecWarps = 8;
 template <typename CT, int V>
 __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
                                                               int n, long long l, float *__restrict__ grad) {
+  pdl_sync();
   __shared__ double as[NGC_MAX_N];
   __shared__ double part[kDecWarps][32 * V];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -176,6 +179,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__rest
 template <typename CT, int V>
 __global__ void __launch_bounds__(256) decode_flat_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
                                                           int n, long long l, float *__restrict__ grad) {
+  pdl_sync();
   __shared__ double as[NGC_MAX_N];
   __shared__ double wt[NGC_MAX_N];
   __shared__ int row[NGC_MAX_N];
@@ -223,18 +227,19 @@ template <typename CT, int V>
 cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, cudaStream_t stream) {
   if (l >= kDecodeFlatFrom) {
     const long long per_block = 256 * V;
-    decode_flat_kernel<CT, V><<<(unsigned)((l + per_block - 1) / per_block), 256, 0, stream>>>(
+    launch_k(decode_flat_kernel<CT, V>, (unsigned)((l + per_block - 1) / per_block), 256, 0, stream, 
         static_cast<const CT *>(coded), a, n, l, grad);
     return cudaGetLastError();
   }
   const long long per_block = 32 * V;
   const unsigned blocks = (unsigned)((l + per_block - 1) / per_block);
-  decode_kernel<CT, V><<<blocks, kDecWarps * 32, 0, stream>>>(static_cast<const CT *>(coded), a, n, l, grad);
+  launch_k(decode_kernel<CT, V>, blocks, kDecWarps * 32, 0, stream, static_cast<const CT *>(coded), a, n, l, grad);
   return cudaGetLastError();
 }
 
 __global__ void __launch_bounds__(256) gd_update_kernel(float *__restrict__ theta, const float *__restrict__ grad,
                                                         long long l, float step) {
+  pdl_sync();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < l) theta[i] = fmaf(-step, grad[i], theta[i]);
 }
@@ -242,7 +247,7 @@ __global__ void __launch_bounds__(256) gd_update_kernel(float *__restrict__ thet
 }  // namespace
 
 cudaError_t launch_gd_update(float *theta, const float *grad, long long l, float step, cudaStream_t stream) {
-  gd_update_kernel<<<(unsigned)((l + 255) / 256), 256, 0, stream>>>(theta, grad, l, step);
+  launch_k(gd_update_kernel, (unsigned)((l + 255) / 256), 256, 0, stream, theta, grad, l, step);
   return cudaGetLastError();
 }
 
@@ -252,7 +257,7 @@ cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *
   const int warps = (batch < kSolveWarps) ? batch : kSolveWarps;
   const unsigned blocks = (unsigned)((batch + warps - 1) / warps);
   const size_t smem = (size_t)warps * solve_warp_bytes(p.n, lv.s);  // at most 4 x 10.3 KB
-  decode_solve_kernel<<<blocks, warps * 32, smem, stream>>>(masks_dev, one, batch, p.n, lv.s, lv.d_a0, lv.d_N,
+  launch_k(decode_solve_kernel, blocks, warps * 32, smem, stream, masks_dev, one, batch, p.n, lv.s, lv.d_a0, lv.d_N,
                                                            lv.d_coef, a_dev, resid_dev, maxres_dev);
   return cudaGetLastError();
 }

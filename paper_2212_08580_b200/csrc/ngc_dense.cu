@@ -12,6 +12,7 @@
 // epilogue (one accumulator row per thread).  Two 256-column accumulators let the epilogue of one
 // tile overlap the contraction of the next.
 #include "ngc_device.h"
+#include "ngc_pdl.cuh"
 #include "ngc_tc.cuh"
 
 namespace ngc {
@@ -159,6 +160,7 @@ __device__ __forceinline__ void transpose_tile_to_bf16(const float *__restrict__
 __global__ void __launch_bounds__(256)
 transpose_to_bf16_kernel(const float *__restrict__ W, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ Wt,
                          int d, int C, int ld) {
+  pdl_sync();
   __shared__ float tile[32][33];
   transpose_tile_to_bf16(W, bias, Wt, d, C, ld, blockIdx.x, blockIdx.y, tile);
 }
@@ -300,6 +302,7 @@ __device__ __forceinline__ void store_staged_tile(const __nv_bfloat16 *stage, __
 template <int EPI>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const Smem s = carve(smem_raw, kFwdStages);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -405,6 +408,7 @@ __global__ void __launch_bounds__(kHeadThreads)
 mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C, const float *__restrict__ W2,
                 const float *__restrict__ b2, const int *__restrict__ y, long long rows_total,
                 __nv_bfloat16 *__restrict__ D1, __nv_bfloat16 *__restrict__ D2) {
+  pdl_sync();
   extern __shared__ __align__(16) unsigned char head_smem[];
   float *w2s = reinterpret_cast<float *>(head_smem);                 // [hidden][CPAD], then b2[CPAD]
   float *zpart = w2s + (size_t)hidden * CPAD + CPAD;                 // [4][kHeadRows][CPAD]
@@ -578,6 +582,7 @@ struct MlpPrepParams {
 };
 
 __global__ void __launch_bounds__(256) mlp_prep_kernel(const MlpPrepParams p) {
+  pdl_sync();
   __shared__ float tile[32][33];
   int b = blockIdx.x;
   if (b < p.tr_blocks) {
@@ -597,6 +602,7 @@ __global__ void __launch_bounds__(kHeadTcThreads, 1)
 mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW2t,
                    const __grid_constant__ CUtensorMap tmW2k, const __grid_constant__ CUtensorMap tmD1,
                    const HeadTcParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char *sm = smem_raw + ((1024u - (base & 1023u)) & 1023u);
@@ -884,6 +890,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
 // bit-identical).  blockIdx.y = partition.
 __global__ void head_reduce_kernel(const float *__restrict__ slots, int max_slots, int wstride, int tpp, int num_tiles,
                                    int grid, float *__restrict__ G, size_t g_batch) {
+  pdl_sync();
   const int j = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= wstride) return;
   // CTAs of the head kernel whose tile range meets partition j
@@ -907,6 +914,7 @@ __global__ void head_reduce_kernel(const float *__restrict__ slots, int max_slot
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kTcThreads, 1)
 tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TnParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const Smem s = carve(smem_raw, kStages);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1068,6 +1076,7 @@ __device__ __forceinline__ void pair_teardown(int warp, uint32_t tmem_base, bool
 template <int EPI>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const PairSmem s = carve_pair(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1160,6 +1169,7 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // Backward contraction on a CTA pair: tile = (batch j, 256 rows of M, 256 columns of N); N must be 256.
 __global__ void __launch_bounds__(kTcThreads, 1)
 tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TnParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const PairSmem s = carve_pair(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1289,6 +1299,7 @@ __host__ __device__ inline void wide_pass_widths(int n_total, int pass, int *w0,
 __global__ void __launch_bounds__(kWideThreads, 1)
 tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const TnWideParams p) {
+  pdl_sync();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = smem_u32(smem_raw);
   unsigned char *tiles = smem_raw + ((1024u - (sbase & 1023u)) & 1023u);
@@ -1425,13 +1436,15 @@ cudaError_t launch_pair(Kern kern, int threads, int pair_tiles, int sms, const C
   cfg.blockDim = dim3(threads);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kern, m0, m1, p);
 }
 
@@ -1505,7 +1518,7 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
     return cudaErrorInvalidValue;
 
   dim3 tg((C + 31) / 32, (d + 31) / 32);
-  transpose_to_bf16_kernel<<<tg, 256, 0, stream>>>(W, nullptr, Wt, d, C, d);
+  launch_k(transpose_to_bf16_kernel, tg, 256, 0, stream, W, nullptr, Wt, d, C, d);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
@@ -1529,7 +1542,7 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   } else {
     p.row_blocks = (rows + 127) / 128;
     p.num_tiles = k * p.row_blocks;
-    fwd_kernel<0><<<p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream>>>(tmXa, tmW, p);
+    launch_k(fwd_kernel<0>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, tmXa, tmW, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
@@ -1546,7 +1559,7 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
     return launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, tmXb, tmR, t, stream);
   }
   t.m_tiles = (d + 127) / 128; t.num_tiles = k * t.m_tiles;
-  tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmR, t);
+  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmXb, tmR, t);
   return cudaGetLastError();
 }
 
@@ -1640,7 +1653,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   pp.tr_bx = (hidden + 31) / 32; pp.tr_blocks = pp.tr_bx * ((dpad + 31) / 32);
   pp.w2_blocks = head_tc ? (hidden * 64 + 255) / 256 : 0;
   const long long groups = (long long)kr * (dpad / 8);
-  mlp_prep_kernel<<<(unsigned)(pp.tr_blocks + pp.w2_blocks + (groups + 255) / 256), 256, 0, stream>>>(pp);
+  launch_k(mlp_prep_kernel, (unsigned)(pp.tr_blocks + pp.w2_blocks + (groups + 255) / 256), 256, 0, stream, pp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
@@ -1663,7 +1676,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     p.num_tiles = k * p.row_blocks * p.n_tiles;
     e = launch_pair(fwd_pair_kernel<1>, kFwdThreads, p.num_tiles, sms, tmXa, tmWh, p, stream);
   } else {
-    fwd_kernel<1><<<p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream>>>(tmXa, tmW, p);
+    launch_k(fwd_kernel<1>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, tmXa, tmW, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
@@ -1682,11 +1695,11 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     e = cudaFuncSetAttribute(mlp_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_tc_smem);
     if (e != cudaSuccess) return e;
     // the same 128 x 64 box serves the loads of h and the stores of delta1
-    mlp_head_tc_kernel<<<hgrid, kHeadTcThreads, head_tc_smem, stream>>>(tmHa, tmW2t, tmW2k, tmD1s, hp);
+    launch_k(mlp_head_tc_kernel, hgrid, kHeadTcThreads, head_tc_smem, stream, tmHa, tmW2t, tmW2k, tmD1s, hp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (fuse_w2) {
       const int wstride = hidden * C + C;
-      head_reduce_kernel<<<dim3((wstride + 255) / 256, k), 256, 0, stream>>>(slots, max_slots, wstride, tpp, k * tpp, hgrid,
+      launch_k(head_reduce_kernel, dim3((wstride + 255) / 256, k), 256, 0, stream, slots, max_slots, wstride, tpp, k * tpp, hgrid,
                                                                             G + (size_t)d * hidden + hidden, lpad);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -1698,7 +1711,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   do {                                                                                                            \
     e = cudaFuncSetAttribute(mlp_head_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem);   \
     if (e != cudaSuccess) return e;                                                                               \
-    mlp_head_kernel<CP><<<head_blocks, kHeadThreads, head_smem, stream>>>(H, hpad, hidden, C, W2, b2, y,          \
+    launch_k(mlp_head_kernel<CP>, head_blocks, kHeadThreads, head_smem, stream, H, hpad, hidden, C, W2, b2, y,          \
                                                                           (long long)kr, D1, D2);                 \
   } while (0)
     if (cpad == 4) NGC_LAUNCH_HEAD(4);
@@ -1724,7 +1737,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     wp.n_total = d + 1; wp.out = G; wp.out_batch = lpad; wp.out_ld = hidden; wp.status = status;
     e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, tmD1, tmXb, wp, stream, kSmemWide);
   } else {
-    tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmXb, tmD1, t);
+    launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmXb, tmD1, t);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess || fuse_w2) return e;
@@ -1733,7 +1746,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   t.N = 16; t.nbox = 1;
   t.m_store = hidden + 1; t.n_store = C;
   t.out = G + (size_t)d * hidden + hidden; t.out_batch = lpad; t.out_ld = C;
-  tn_gemm_kernel<<<t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream>>>(tmH, tmD2, t);
+  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmH, tmD2, t);
   return cudaGetLastError();
 }
 

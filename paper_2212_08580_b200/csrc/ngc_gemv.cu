@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include "ngc_device.h"
+#include "ngc_pdl.cuh"
 #include "ngc_f32x2.cuh"
 
 namespace ngc {
@@ -160,6 +161,7 @@ template <> struct Log2<8> { static constexpr int v = 3; };
 
 template <typename XT, int VPT, int R, int ACT>
 __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams p) {
+  pdl_sync();
   constexpr int VN = Vec<XT>::N;
   constexpr int VH = VN / 2;  // packed pairs per vector
   extern __shared__ __align__(128) unsigned char smem[];
@@ -324,7 +326,7 @@ cudaError_t launch_one(const GemvParams &p, cudaStream_t stream) {
   auto kern = gemv_pair_kernel<XT, VPT, R, ACT>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<p.split.grid, kThreads, smem, stream>>>(p);
+  launch_k(kern, p.split.grid, kThreads, smem, stream, p);
   return cudaGetLastError();
 }
 
@@ -422,6 +424,7 @@ template <typename CT>
 __global__ void __launch_bounds__(kEncWarps * 32)
 combine_encode_kernel(const RowSplit split, const float *__restrict__ ws, const double *__restrict__ coef, int n, int s,
                       int d, CT *__restrict__ coded, int kEncRows /* workers per block */) {
+  pdl_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int held = min(kEncRows + s, n);
   double *Gs = reinterpret_cast<double *>(smem_raw);            // [held][kEncCols]
@@ -487,6 +490,7 @@ template <typename CT, int S1>
 __global__ void __launch_bounds__(128)
 encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n,
                      long long d, int chunk, CT *__restrict__ coded) {
+  pdl_sync();
   constexpr int W = S1 + kEncLook;
   __shared__ CT cs[NGC_MAX_N * S1];
   const int first = blockIdx.y * chunk;
@@ -575,6 +579,7 @@ template <typename CT>
 __global__ void __launch_bounds__(256)
 encode_simple_kernel(const RowSplit split, const float *__restrict__ ws, long long ld_ws,
                      const double *__restrict__ coef, int n, int s, long long d, CT *__restrict__ coded) {
+  pdl_sync();
   const long long col = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (col >= d) return;
   for (int i = 0; i < n; ++i) {
@@ -618,7 +623,7 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
                               long long d, CT *coded, cudaStream_t stream) {
   EncodeKernel<CT> kern = (split.P == 1 && s + 1 <= kEncMaxS1) ? encode_window_for<CT>(s + 1) : nullptr;
   if (!kern) {
-    encode_simple_kernel<CT><<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(split, ws, ld_ws, coef, n, s, d, coded);
+    launch_k(encode_simple_kernel<CT>, (unsigned)((d + 255) / 256), 256, 0, stream, split, ws, ld_ws, coef, n, s, d, coded);
     return cudaGetLastError();
   }
   // Number of worker chunks: the blocks run in rounds of `capacity` resident blocks, a block's time grows
@@ -638,7 +643,7 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
   }
   const int chunk = (n + best_chunks - 1) / best_chunks;
   const dim3 grid((unsigned)col_blocks, (unsigned)((n + chunk - 1) / chunk));
-  kern<<<grid, 128, 0, stream>>>(ws, ld_ws, coef, n, d, chunk, coded);
+  launch_k(kern, grid, 128, 0, stream, ws, ld_ws, coef, n, d, chunk, coded);
   return cudaGetLastError();
 }
 }  // namespace
@@ -666,12 +671,12 @@ cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const 
   if (coded_dtype == NGC_F64) {
     e = cudaFuncSetAttribute(combine_encode_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    combine_encode_kernel<double><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
+    launch_k(combine_encode_kernel<double>, grid, kEncWarps * 32, smem, stream, split, ws, d_coef, n, s, d,
                                                                           static_cast<double *>(coded), enc_rows);
   } else {
     e = cudaFuncSetAttribute(combine_encode_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    combine_encode_kernel<float><<<grid, kEncWarps * 32, smem, stream>>>(split, ws, d_coef, n, s, d,
+    launch_k(combine_encode_kernel<float>, grid, kEncWarps * 32, smem, stream, split, ws, d_coef, n, s, d,
                                                                          static_cast<float *>(coded), enc_rows);
   }
   return cudaGetLastError();

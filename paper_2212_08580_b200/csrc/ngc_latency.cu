@@ -4,6 +4,7 @@
 #include <cmath>
 
 #include "ngc_device.h"
+#include "ngc_pdl.cuh"
 
 namespace ngc {
 namespace {
@@ -26,6 +27,7 @@ struct McParams {
 };
 
 __global__ void __launch_bounds__(128) latency_mc_kernel(const McParams p) {
+  pdl_sync();
   const long long trial = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (trial >= p.trials) return;
   const uint64_t seed = splitmix64_at(p.seed ^ 0xD1B54A32D192ED03ull, (uint64_t)trial + 1);
@@ -76,7 +78,7 @@ cudaError_t launch_latency_mc(const ngc_plan_s &plan, uint64_t seed, long long t
   p.seed = seed; p.trials = trials; p.shift = shift; p.rate = rate; p.p_fail = p_fail;
   p.gamma = plan.gamma; p.eps = plan.eps;
   p.latency = latency_dev; p.level = level_dev;
-  latency_mc_kernel<<<(unsigned)((trials + 127) / 128), 128, 0, stream>>>(p);
+  launch_k(latency_mc_kernel, (unsigned)((trials + 127) / 128), 128, 0, stream, p);
   return cudaGetLastError();
 }
 
