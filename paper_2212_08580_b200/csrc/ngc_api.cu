@@ -148,6 +148,7 @@ void ngc_plan_destroy(ngc_plan_t *p) {
     cudaFree(p->d_masks);
     cudaFree(p->d_status);
     cudaFree(p->d_maxres);
+    cudaFree(p->d_gpart);
     cudaFree(p->st_X);
     cudaFree(p->st_y);
     cudaFree(p->st_theta);
@@ -161,8 +162,54 @@ void ngc_plan_destroy(ngc_plan_t *p) {
   delete p;
 }
 
+}  // extern "C"
+
+namespace {
+
+// What ngc_step hands to the gradient + encode launcher so that the decode can ride on the encode kernel
+// of the dense models: the event after which the decoding vector is on the device, where the decoded
+// gradient goes, and whether the encode took the decode along.
+struct DecodeHook {
+  cudaEvent_t solved;
+  float *grad;
+  bool fused;
+};
+
+int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
+                     void *coded, void *cuda_stream, DecodeHook *hook);
+
+}  // namespace
+
+extern "C" {
+
 int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
                     void *coded, void *cuda_stream) {
+  return grad_encode_impl(p, m, theta, X, y, layer, coded, cuda_stream, nullptr);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Encode of a dense model's partial gradients; with a hook, the decode in the same kernel.
+int encode_dense(ngc_plan_t *p, const ngc::RowSplit &split, const float *G, long long ldG, const ngc_level_t &lv,
+                 long long l, void *coded, int cdt, cudaStream_t stream, DecodeHook *hook) {
+  if (!hook) {
+    NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, l, coded, cdt, stream));
+    return NGC_OK;
+  }
+  const int rc = ensure_staging(p, &p->d_gpart, &p->gpart_bytes, (size_t)ngc::kEncodeMaxChunks * l * sizeof(double));
+  if (rc != NGC_OK) return rc;
+  NGC_CUDA(p, cudaStreamWaitEvent(stream, hook->solved, 0));
+  ngc::EncodeDecodeArgs dec{p->d_a, static_cast<double *>(p->d_gpart), hook->grad, &hook->fused};
+  NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, l, coded, cdt, stream, &dec));
+  if (hook->fused) p->launches += 1;  // the sum over the worker chunks
+  return NGC_OK;
+}
+
+int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
+                     void *coded, void *cuda_stream, DecodeHook *hook) {
+  if (hook) hook->fused = false;
   if (!p || !theta || !X || !y || !coded || layer < 0 || layer >= p->L) return NGC_ERR_INVALID;
   int rc = check_model(p, m);
   if (rc != NGC_OK) return rc;
@@ -207,7 +254,7 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     ngc::RowSplit split;
     split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
     const long long l = ngc_num_params(m);
-    NGC_CUDA(p, ngc::launch_encode_long(split, G, l, lv.d_coef, p->n, lv.s, l, coded, cdt, stream));
+    if ((rc = encode_dense(p, split, G, l, lv, l, coded, cdt, stream, hook)) != NGC_OK) return rc;
     p->launches += 4;
     return NGC_OK;
   }
@@ -229,12 +276,16 @@ int ngc_grad_encode(ngc_plan_t *p, const ngc_model_t *m, const void *theta, cons
     if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     ngc::RowSplit split;
     split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
-    NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, ngc_num_params(m), coded, cdt, stream));
+    if ((rc = encode_dense(p, split, G, ldG, lv, ngc_num_params(m), coded, cdt, stream, hook)) != NGC_OK) return rc;
     p->launches += ngc::mlp_launch_count(h);
     return NGC_OK;
   }
   return NGC_ERR_INVALID;
 }
+
+}  // namespace
+
+extern "C" {
 
 int ngc_decode_vectors(ngc_plan_t *p, int layer, const int32_t *S, int nS, int batch, double *a_out,
                        double *resid_out) {
@@ -335,12 +386,17 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
   NGC_CUDA(p, cudaStreamWaitEvent(side, decoded, 0));
   NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
   NGC_CUDA(p, cudaEventRecord(solved, side));
-  rc = ngc_grad_encode(p, m, theta, X, y, info->layer, coded, cuda_stream);
+  // Dense models: the encode kernel forms the decoded gradient from the coded rows as it writes them.
+  DecodeHook hook{solved, grad, false};
+  rc = grad_encode_impl(p, m, theta, X, y, info->layer, coded, cuda_stream, &hook);
   if (rc != NGC_OK) return rc;
-  NGC_CUDA(p, cudaStreamWaitEvent(stream, solved, 0));
-  NGC_CUDA(p, ngc::launch_decode(coded, ngc_coded_dtype(p, m), p->d_a, p->n, ngc_num_params(m), grad, stream));
+  if (!hook.fused) {
+    NGC_CUDA(p, cudaStreamWaitEvent(stream, solved, 0));
+    NGC_CUDA(p, ngc::launch_decode(coded, ngc_coded_dtype(p, m), p->d_a, p->n, ngc_num_params(m), grad, stream));
+    p->launches += 1;
+  }
   NGC_CUDA(p, cudaEventRecord(decoded, stream));
-  p->launches += 2;
+  p->launches += 1;  // the solve
   return NGC_OK;
 }
 
@@ -388,7 +444,8 @@ int ngc_gd_update(float *theta, const float *grad, int64_t l, float step, void *
 
 size_t ngc_workspace_bytes(const ngc_plan_t *p) {
   if (!p) return 0;
-  return p->ws_bytes + p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes + p->st_grad_bytes;
+  return p->ws_bytes + p->gpart_bytes + p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes +
+         p->st_grad_bytes;
 }
 
 int ngc_device_status(ngc_plan_t *p, double *residual_out) {

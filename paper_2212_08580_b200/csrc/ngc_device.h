@@ -46,12 +46,24 @@ cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *
 cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
                           cudaStream_t stream);
 
-// Same encode for long gradients (dense models): every partial gradient is read once, windows live in
-// registers.  ws is [group][slot][ld_ws] fp32, ld_ws a multiple of 4 and >= d.
 // True when an SM that holds a CTA of the gradient kernel chosen for `m` can still take a one-warp block.
 bool gemv_pair_leaves_room(const ngc_model_t &m);
+
+// Same encode for long gradients (dense models): every partial gradient is read once, windows live in
+// registers.  ws is [group][slot][ld_ws] fp32, ld_ws a multiple of 4 and >= d.
+// With `dec` (and a window that fits the register ring) the decode rides along: the kernel also forms
+// grad = sum_i a[i] * coded[i] from the values it has just produced, through `gpart` (kEncodeMaxChunks x d
+// doubles of scratch); *fused tells whether it did.
+constexpr int kEncodeMaxChunks = 16;
+struct EncodeDecodeArgs {
+  const double *a;  // decoding vector on the device, n weights, zero outside the responsive set
+  double *gpart;
+  float *grad;
+  bool *fused;
+};
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
-                               int s, long long d, void *coded, int coded_dtype, cudaStream_t stream);
+                               int s, long long d, void *coded, int coded_dtype, cudaStream_t stream,
+                               const EncodeDecodeArgs *dec = nullptr);
 
 // MLP (one hidden ReLU layer, softmax cross-entropy) partial gradients on the tensor cores (X fp32):
 // G[k][*G_ld] fp32 inside `scratch`, each row holding [dW1, db1, dW2, db2].

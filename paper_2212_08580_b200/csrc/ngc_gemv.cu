@@ -485,18 +485,27 @@ namespace {
 // chunks overlap by s groups, which come from L2.
 constexpr int kEncLook = 6;
 constexpr int kEncMaxS1 = 12;
+constexpr int kEncMaxChunks = kEncodeMaxChunks;
 
-template <typename CT, int S1>
+// DEC: the decode rides along.  `avec` is the decoding vector (n weights, zero for workers outside the
+// responsive set); each thread also forms sum_i avec[i] * x_i over its chunk of workers from the coded values
+// exactly as they are stored, in fp64, and leaves it in gpart[chunk index][d] for `decode_sum_kernel`: the
+// coded matrix is not read a second time.
+template <typename CT, int S1, bool DEC>
 __global__ void __launch_bounds__(128)
 encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n,
-                     long long d, int chunk, CT *__restrict__ coded) {
+                     long long d, int chunk, CT *__restrict__ coded, const double *__restrict__ avec,
+                     double *__restrict__ gpart) {
   pdl_sync();
   constexpr int W = S1 + kEncLook;
   __shared__ CT cs[NGC_MAX_N * S1];
+  __shared__ double as[DEC ? NGC_MAX_N : 1];
   const int first = blockIdx.y * chunk;
   const int last = (first + chunk < n) ? first + chunk : n;  // workers first .. last-1
   if (first >= last) return;
   for (int e = threadIdx.x; e < (last - first) * S1; e += 128) cs[e] = (CT)coef[(size_t)first * S1 + e];
+  if constexpr (DEC)
+    for (int e = threadIdx.x; e < last - first; e += 128) as[e] = avec[first + e];
   __syncthreads();
   const long long col = ((long long)blockIdx.x * 128 + threadIdx.x) * 4;
   if (col >= d) return;
@@ -514,6 +523,7 @@ encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double
   const int store_mode = (d % 4 == 0) ? 4 : (d % 2 == 0) ? 2 : 1;
   const CT *ci = cs;
   CT *dst = coded + (size_t)first * d + col;
+  double gacc[4] = {0.0, 0.0, 0.0, 0.0};
   for (int i0 = first; i0 < last; i0 += W) {
 #pragma unroll
     for (int t = 0; t < W; ++t) {
@@ -563,6 +573,13 @@ encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double
           if (col + 2 < d) dst[2] = out[2];
           if (col + 3 < d) dst[3] = out[3];
         }
+        if constexpr (DEC) {
+          const double ai = as[i0 + t - first];
+          if (ai != 0.0) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) gacc[e] = fma(ai, (double)out[e], gacc[e]);
+          }
+        }
         ci += S1;
         dst += d;
         // the oldest group is no longer needed; its slot takes the next group of the chunk, if any is left
@@ -572,6 +589,29 @@ encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double
       }
     }
   }
+  if constexpr (DEC) {
+    double *gp = gpart + (size_t)blockIdx.y * d + col;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (col + e < d) gp[e] = gacc[e];
+  }
+}
+
+// grad = sum over the worker chunks of the partial decodes, in chunk order.
+__global__ void __launch_bounds__(256) decode_sum_kernel(const double *__restrict__ gpart, int chunks, long long d,
+                                                         float *__restrict__ grad) {
+  pdl_sync();
+  const long long col = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= d) return;
+  double acc = 0.0;
+  for (int c0 = 0; c0 < chunks; c0 += 4) {
+    double v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = c0 + i < chunks ? gpart[(size_t)(c0 + i) * d + col] : 0.0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc += v[i];
+  }
+  grad[col] = (float)acc;
 }
 
 // Plain fallback (very wide windows): one thread per column.
@@ -597,31 +637,34 @@ encode_simple_kernel(const RowSplit split, const float *__restrict__ ws, long lo
 }
 
 template <typename CT>
-using EncodeKernel = void (*)(const float *, long long, const double *, int, long long, int, CT *);
+using EncodeKernel = void (*)(const float *, long long, const double *, int, long long, int, CT *, const double *, double *);
 
-template <typename CT>
+template <typename CT, bool DEC>
 EncodeKernel<CT> encode_window_for(int s1) {
   switch (s1) {
-    case 1: return encode_window_kernel<CT, 1>;
-    case 2: return encode_window_kernel<CT, 2>;
-    case 3: return encode_window_kernel<CT, 3>;
-    case 4: return encode_window_kernel<CT, 4>;
-    case 5: return encode_window_kernel<CT, 5>;
-    case 6: return encode_window_kernel<CT, 6>;
-    case 7: return encode_window_kernel<CT, 7>;
-    case 8: return encode_window_kernel<CT, 8>;
-    case 9: return encode_window_kernel<CT, 9>;
-    case 10: return encode_window_kernel<CT, 10>;
-    case 11: return encode_window_kernel<CT, 11>;
-    case 12: return encode_window_kernel<CT, 12>;
+    case 1: return encode_window_kernel<CT, 1, DEC>;
+    case 2: return encode_window_kernel<CT, 2, DEC>;
+    case 3: return encode_window_kernel<CT, 3, DEC>;
+    case 4: return encode_window_kernel<CT, 4, DEC>;
+    case 5: return encode_window_kernel<CT, 5, DEC>;
+    case 6: return encode_window_kernel<CT, 6, DEC>;
+    case 7: return encode_window_kernel<CT, 7, DEC>;
+    case 8: return encode_window_kernel<CT, 8, DEC>;
+    case 9: return encode_window_kernel<CT, 9, DEC>;
+    case 10: return encode_window_kernel<CT, 10, DEC>;
+    case 11: return encode_window_kernel<CT, 11, DEC>;
+    case 12: return encode_window_kernel<CT, 12, DEC>;
     default: return nullptr;
   }
 }
 
 template <typename CT>
 cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long ld_ws, const double *coef, int n, int s,
-                              long long d, CT *coded, cudaStream_t stream) {
-  EncodeKernel<CT> kern = (split.P == 1 && s + 1 <= kEncMaxS1) ? encode_window_for<CT>(s + 1) : nullptr;
+                              long long d, CT *coded, cudaStream_t stream, const EncodeDecodeArgs *dec) {
+  const bool window = split.P == 1 && s + 1 <= kEncMaxS1;
+  const bool fuse = window && dec && dec->a && dec->gpart && dec->grad;
+  if (dec && dec->fused) *dec->fused = fuse;
+  EncodeKernel<CT> kern = !window ? nullptr : (fuse ? encode_window_for<CT, true>(s + 1) : encode_window_for<CT, false>(s + 1));
   if (!kern) {
     launch_k(encode_simple_kernel<CT>, (unsigned)((d + 255) / 256), 256, 0, stream, split, ws, ld_ws, coef, n, s, d, coded);
     return cudaGetLastError();
@@ -635,7 +678,7 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
   const long long col_blocks = (d + 511) / 512;
   int best_chunks = 1;
   long long best_cost = -1;
-  for (int chunks = 1; chunks <= n && chunks <= 16; ++chunks) {
+  for (int chunks = 1; chunks <= n && chunks <= kEncMaxChunks; ++chunks) {
     const int chunk = (n + chunks - 1) / chunks;
     const long long blocks = col_blocks * ((n + chunk - 1) / chunk);
     const long long cost = ((blocks + capacity - 1) / capacity) * (chunk + s + 4);
@@ -643,18 +686,23 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
   }
   const int chunk = (n + best_chunks - 1) / best_chunks;
   const dim3 grid((unsigned)col_blocks, (unsigned)((n + chunk - 1) / chunk));
-  launch_k(kern, grid, 128, 0, stream, ws, ld_ws, coef, n, d, chunk, coded);
+  launch_k(kern, grid, 128, 0, stream, ws, ld_ws, coef, n, d, chunk, coded, fuse ? dec->a : nullptr,
+           fuse ? dec->gpart : nullptr);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess || !fuse) return err;
+  launch_k(decode_sum_kernel, (unsigned)((d + 255) / 256), 256, 0, stream, dec->gpart, (int)grid.y, d, dec->grad);
   return cudaGetLastError();
 }
 }  // namespace
 
 // Encode for the dense models: ws holds [group][slot][ld_ws] fp32, every slot filled, ld_ws a multiple of 4 and >= d.
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
-                               int s, long long d, void *coded, int coded_dtype, cudaStream_t stream) {
+                               int s, long long d, void *coded, int coded_dtype, cudaStream_t stream,
+                               const EncodeDecodeArgs *dec) {
   if (ld_ws % 4 != 0 || ld_ws < d) return cudaErrorInvalidValue;
   if (coded_dtype == NGC_F64)
-    return encode_long_typed<double>(split, ws, ld_ws, d_coef, n, s, d, static_cast<double *>(coded), stream);
-  return encode_long_typed<float>(split, ws, ld_ws, d_coef, n, s, d, static_cast<float *>(coded), stream);
+    return encode_long_typed<double>(split, ws, ld_ws, d_coef, n, s, d, static_cast<double *>(coded), stream, dec);
+  return encode_long_typed<float>(split, ws, ld_ws, d_coef, n, s, d, static_cast<float *>(coded), stream, dec);
 }
 
 cudaError_t launch_combine_encode(const RowSplit &split, const float *ws, const double *d_coef, int n, int s, int d,
