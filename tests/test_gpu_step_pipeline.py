@@ -43,3 +43,33 @@ def test_queued_steps_each_use_their_own_decoding_vector(name, rows, tol):
     for it in ran:
         assert rel_l2(got[it], g_full) < tol, it
     assert p.device_status() < 1e-6
+
+
+@pytest.mark.parametrize("name,rows", [("softmax50", 300), ("mlp30", 200)])
+def test_step_of_a_dense_model_matches_encode_then_decode(name, rows):
+    """ngc_step lets the decode ride on the encode kernel of the dense models; ngc_grad_encode followed by
+    ngc_decode reads the coded matrix back.  Same coded rows bit for bit, same decoded gradient up to the
+    order of the fp64 sums."""
+    w = replace(ngc_inputs.shrink(ngc_inputs.WORKLOADS[name], rows=rows), pattern="sets")
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    l = w.n_params
+    cdt = p.coded_dtype(m)
+    coded_a = torch.empty((w.n, l), dtype=coded_torch_dtype(cdt), device="cuda")
+    coded_b = torch.empty_like(coded_a)
+    grad_a = torch.empty(l, dtype=torch.float32, device="cuda")
+    grad_b = torch.empty_like(grad_a)
+    for it in (0, 3, 7, 10):                                      # straggler sets of different sizes: several levels
+        t = ngc_inputs.pattern_times(w, it)
+        coded_a.fill_(float("nan"))
+        grad_a.fill_(float("nan"))
+        info = p.step(m, theta, X, y, t, coded_a, grad_a)
+        p.grad_encode(m, theta, X, y, info.layer, coded_b)
+        p.decode(info.layer, info.responsive(), coded_b, cdt, l, grad_b)
+        torch.cuda.synchronize()
+        assert torch.equal(coded_a, coded_b)
+        ga, gb = grad_a.cpu().numpy(), grad_b.cpu().numpy()
+        assert np.isfinite(ga).all()
+        assert rel_l2(ga, gb) < 1e-6, (it, info.layer, rel_l2(ga, gb))
+    assert p.device_status() < 1e-6
