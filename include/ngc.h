@@ -166,7 +166,13 @@ int ngc_decode(ngc_plan_t *plan, int layer, const int32_t *S_host, int nS, const
 /*
  * One full iteration for a given straggler pattern: ngc_select on the host, then
  * ngc_grad_encode for the chosen component and ngc_decode over its responsive set,
- * enqueued on the stream.  coded_dev is caller-provided scratch of n x l coded values.
+ * enqueued on the stream.  coded_dev is caller-provided scratch of n x l coded values; it
+ * holds the workers' coded gradients x_i afterwards, as ngc_grad_encode would leave them.
+ * The responsive set is known before any gradient is, so the decoding vector is solved on
+ * a stream of the plan's own while the gradients are computed, and for the softmax and
+ * MLP models the weighted sum of the decode is formed by the encode kernel from the coded
+ * values as it writes them (same result as ngc_decode up to the order of its fp64 sums).
+ * The first call for a model allocates the plan's scratch (ngc_workspace_bytes).
  */
 int ngc_step(ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev, const void *X_dev,
              const void *y_dev, const double *task_times_host, void *coded_dev, float *grad_dev,
