@@ -333,7 +333,14 @@ int ngc_decode(ngc_plan_t *p, int layer, const int32_t *S, int nS, const void *c
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
   NGC_CUDA(p, ngc::launch_decode(coded, coded_dtype, p->d_a, p->n, l, grad, stream));
-  if (p->ev_decoded) NGC_CUDA(p, cudaEventRecord(static_cast<cudaEvent_t>(p->ev_decoded), stream));
+  if (p->ev_decoded) {
+    // tells the side stream of ngc_step that the vector has been read; an event recorded inside a stream
+    // capture could not be waited for by the eager steps that follow, and a captured step is in order anyway
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    NGC_CUDA(p, cudaStreamIsCapturing(stream, &cap));
+    if (cap == cudaStreamCaptureStatusNone)
+      NGC_CUDA(p, cudaEventRecord(static_cast<cudaEvent_t>(p->ev_decoded), stream));
+  }
   p->launches += 2;
   return NGC_OK;
 }

@@ -76,3 +76,55 @@ def test_gradient_descent_follows_the_oracle():
     torch.cuda.synchronize()
     assert rel_l2(th.cpu().numpy(), th_o) < 1e-5
     assert all(b < a for a, b in zip(losses, losses[1:]))      # the loss goes down every iteration
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,rows,tol", [("logistic20", 128, 1e-5), ("mlp30", 200, 1e-2)])
+def test_gradient_descent_iteration_replayed_from_a_cuda_graph(name, rows, tol):
+    """One iteration (ngc_step for a fixed straggler pattern + the update of Eq. 1) captured into a CUDA graph
+    and replayed: every replay must do what the eager calls do on the parameters as they then stand, and the
+    plan must stay usable for eager steps afterwards."""
+    from dataclasses import replace
+    w = replace(ngc_inputs.shrink(ngc_inputs.WORKLOADS[name], rows=rows), pattern="sets")
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    l = w.n_params
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    cdt = p.coded_dtype(m)
+    coded = torch.empty((w.n, l), dtype=torch.float64 if cdt == ngc.NGC_F64 else torch.float32, device="cuda")
+    grad = torch.empty(l, dtype=torch.float32, device="cuda")
+    t = ngc_inputs.set_times(w.n, w.levels[-1] + 1, [1, 4])
+    eta = 1e-3 / (w.n * w.rows)
+
+    def eager(th, steps):
+        th = th.clone()
+        for _ in range(steps):
+            p.step(m, th, X, y, t, coded, grad)
+            ngc.gd_update(th, grad, eta)
+        torch.cuda.synchronize()
+        return th
+
+    want1, want3 = eager(theta, 1), eager(theta, 3)       # also allocates everything the plan needs
+    th = theta.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        s = torch.cuda.current_stream().cuda_stream
+        p.step(m, th, X, y, t, coded, grad, s)
+        ngc.gd_update(th, grad, eta, s)
+    torch.cuda.synchronize()
+    assert torch.equal(th, theta)                         # capture runs nothing
+    graph.replay()
+    torch.cuda.synchronize()
+    assert rel_l2(th.cpu().numpy(), want1.cpu().numpy()) < 1e-6
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert rel_l2(th.cpu().numpy(), want3.cpu().numpy()) < 1e-6
+    # eager steps on the same plan still work, and decode the full gradient
+    info = p.step(m, theta, X, y, t, coded, grad)
+    torch.cuda.synchronize()
+    g_full = orc.full_gradient(w.kind, to_np64(X), to_np64(y), to_np64(theta), w.hidden, w.n_classes)
+    assert info.sigma == 2 and rel_l2(grad.cpu().numpy(), g_full) < tol
+    assert p.device_status() < 1e-6
