@@ -73,3 +73,33 @@ def test_step_of_a_dense_model_matches_encode_then_decode(name, rows):
         assert np.isfinite(ga).all()
         assert rel_l2(ga, gb) < 1e-6, (it, info.layer, rel_l2(ga, gb))
     assert p.device_status() < 1e-6
+
+
+def test_one_plan_serves_models_of_growing_and_changing_kind():
+    """The plan's scratch grows with the model it is asked to serve and its choice of decode path follows the
+    model: least squares, then a larger logistic model, softmax regression, an MLP, and least squares again."""
+    n, levels = 6, (1, 2)
+    p = ngc.Plan(n, levels, seed=77)
+    cases = [
+        ngc_inputs.Workload("mix_lsq", 950, n, levels, "lsq", 64, 128, "f32", pattern="sets", unit_x=True),
+        ngc_inputs.Workload("mix_logistic", 951, n, levels, "logistic", 300, 2048, "f32", pattern="sets"),
+        ngc_inputs.Workload("mix_softmax", 952, n, levels, "softmax", 300, 256, "bf16", n_classes=256, pattern="sets"),
+        ngc_inputs.Workload("mix_mlp", 953, n, levels, "mlp", 260, 64, "f32", n_classes=10, hidden=128, pattern="sets"),
+        ngc_inputs.Workload("mix_lsq", 950, n, levels, "lsq", 64, 128, "f32", pattern="sets", unit_x=True),
+    ]
+    seen = 0
+    for it, w in enumerate(cases):
+        X, y, theta = ngc_inputs.make_data(w, "cuda")
+        m = model_of(w)
+        l = w.n_params
+        coded = torch.empty((n, l), dtype=coded_torch_dtype(p.coded_dtype(m)), device="cuda")
+        grad = torch.empty(l, dtype=torch.float32, device="cuda")
+        t = ngc_inputs.set_times(n, levels[-1] + 1, list(range(it % 3)))
+        info = p.step(m, theta, X, y, t, coded, grad)             # queued behind the previous model's step
+        torch.cuda.synchronize()
+        g_full = oracle_G(w, X, y, theta).sum(axis=0)
+        tol = 1e-5 if w.kind in ("lsq", "logistic") else 1e-2
+        assert rel_l2(grad.cpu().numpy(), g_full) < tol, (w.name, info.layer)
+        assert p.workspace_bytes() >= seen
+        seen = p.workspace_bytes()
+    assert p.device_status() < 1e-6
