@@ -103,3 +103,25 @@ def test_one_plan_serves_models_of_growing_and_changing_kind():
         assert p.workspace_bytes() >= seen
         seen = p.workspace_bytes()
     assert p.device_status() < 1e-6
+
+
+@pytest.mark.parametrize("name,rows", [("softmax50", 520), ("mlp30", 2000)])
+def test_dense_steps_are_bitwise_reproducible(name, rows):
+    """Nothing in the dense paths is added up in an order that depends on timing: per-CTA slots and worker
+    chunks are summed in index order.  mlp30 at its full row count has partitions shared by several CTAs of
+    the head kernel and CTAs that carry their sums across tiles."""
+    w = replace(ngc_inputs.shrink(ngc_inputs.WORKLOADS[name], rows=rows), pattern="sets")
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    l = w.n_params
+    t = ngc_inputs.set_times(w.n, w.levels[-1] + 1, [0, 2, 5])
+    outs = []
+    for _ in range(3):
+        coded = torch.empty((w.n, l), dtype=coded_torch_dtype(p.coded_dtype(m)), device="cuda")
+        grad = torch.empty(l, dtype=torch.float32, device="cuda")
+        p.step(m, theta, X, y, t, coded, grad)
+        torch.cuda.synchronize()
+        outs.append((coded.cpu(), grad.cpu()))
+    for c, g in outs[1:]:
+        assert torch.equal(c, outs[0][0]) and torch.equal(g, outs[0][1])
