@@ -93,9 +93,11 @@ def algorithmic_flops(w: ngc_inputs.Workload) -> int:
     return w.n * w.rows * (4 * w.d * w.hidden + 6 * w.hidden * w.n_classes)
 
 
-# dram__bytes_read + dram__bytes_write of the dominant kernel per full-size launch, from the ncu captures
-# summarised under profiles/ (None = not captured for the kernel as it stands).
-TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000}
+# dram__bytes_read + dram__bytes_write per full-size launch of the timed kernel (the dense workloads: summed over the
+# gradient kernels the events bracket), from the ncu captures summarised under profiles/ (None = not captured for
+# the kernels as they stand).
+TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000,
+                 "softmax50": 1_075_000_000, "mlp30": 643_000_000}
 FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
 
 
