@@ -128,3 +128,31 @@ def test_gradient_descent_iteration_replayed_from_a_cuda_graph(name, rows, tol):
     g_full = orc.full_gradient(w.kind, to_np64(X), to_np64(y), to_np64(theta), w.hidden, w.n_classes)
     assert info.sigma == 2 and rel_l2(grad.cpu().numpy(), g_full) < tol
     assert p.device_status() < 1e-6
+
+
+@pytest.mark.gpu
+def test_nested_code_never_waits_longer_than_a_fixed_code_on_the_same_times():
+    """Section III: with negligible signalling time a nested code with levels 0..s_bar stops, in every iteration,
+    as early as the best fixed code does on the same task times, and its responders compute no more than that
+    code's load; gradient descent ends at the same parameters whichever code decodes the gradients."""
+    from paper_2212_08580_b200 import gd_loop
+    n, s_bar, iters = 8, 3, 12
+    w = ngc_inputs.Workload("gd_compare", 902, n, (0,), "lsq", 128, 128, "f32", unit_x=True)
+    X, y, theta0 = ngc_inputs.make_data(w, "cuda")
+    step = 0.5 / (n * w.rows)
+    hist, finals = {}, {}
+    for name, levels in [("nested", list(range(s_bar + 1)))] + [(s, [s]) for s in range(s_bar + 1)]:
+        plan = ngc.Plan(n, levels, seed=5, gamma=0.0, eps=0.0)
+        th = theta0.clone()
+        hist[name] = gd_loop.run(plan, model_of(w), th, X, y, iters, step, seed=4242, rho=0.5, lam=0.5, p_fail=0.0,
+                                 times_width=s_bar + 1)
+        torch.cuda.synchronize()
+        finals[name] = th.cpu().numpy()
+    for it in range(iters):
+        best = min(hist[s].latency[it] for s in range(s_bar + 1))
+        assert hist["nested"].latency[it] == best                      # same times, same arithmetic: equal, not just close
+        s_used = hist["nested"].level[it]                              # level index = tolerance for levels 0..s_bar
+        assert hist[s_used].latency[it] == best
+    assert hist["nested"].total_latency <= min(hist[s].total_latency for s in range(s_bar + 1))
+    for s in range(s_bar + 1):
+        assert rel_l2(finals[s], finals["nested"]) < 1e-5
