@@ -201,9 +201,10 @@ int encode_dense(ngc_plan_t *p, const ngc::RowSplit &split, const float *G, long
   const int rc = ensure_staging(p, &p->d_gpart, &p->gpart_bytes, (size_t)ngc::kEncodeMaxChunks * l * sizeof(double));
   if (rc != NGC_OK) return rc;
   NGC_CUDA(p, cudaStreamWaitEvent(stream, hook->solved, 0));
-  ngc::EncodeDecodeArgs dec{p->d_a, static_cast<double *>(p->d_gpart), hook->grad, &hook->fused};
+  int sum_launches = 0;
+  ngc::EncodeDecodeArgs dec{p->d_a, static_cast<double *>(p->d_gpart), hook->grad, &hook->fused, &sum_launches};
   NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, l, coded, cdt, stream, &dec));
-  if (hook->fused) p->launches += 1;  // the sum over the worker chunks
+  p->launches += sum_launches;  // the sum over the worker chunks, when there are several
   return NGC_OK;
 }
 

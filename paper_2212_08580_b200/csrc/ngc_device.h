@@ -53,13 +53,14 @@ bool gemv_pair_leaves_room(const ngc_model_t &m);
 // registers.  ws is [group][slot][ld_ws] fp32, ld_ws a multiple of 4 and >= d.
 // With `dec` (and a window that fits the register ring) the decode rides along: the kernel also forms
 // grad = sum_i a[i] * coded[i] from the values it has just produced, through `gpart` (kEncodeMaxChunks x d
-// doubles of scratch); *fused tells whether it did.
+// doubles of scratch) when the workers are cut into several chunks; *fused tells whether it did.
 constexpr int kEncodeMaxChunks = 16;
 struct EncodeDecodeArgs {
   const double *a;  // decoding vector on the device, n weights, zero outside the responsive set
   double *gpart;
   float *grad;
   bool *fused;
+  int *sum_launches;  // out: 1 when the chunk sum ran as a kernel of its own (more than one worker chunk), else 0
 };
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
                                int s, long long d, void *coded, int coded_dtype, cudaStream_t stream,

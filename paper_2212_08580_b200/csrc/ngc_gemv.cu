@@ -489,13 +489,13 @@ constexpr int kEncMaxChunks = kEncodeMaxChunks;
 
 // DEC: the decode rides along.  `avec` is the decoding vector (n weights, zero for workers outside the
 // responsive set); each thread also forms sum_i avec[i] * x_i over its chunk of workers from the coded values
-// exactly as they are stored, in fp64, and leaves it in gpart[chunk index][d] for `decode_sum_kernel`: the
-// coded matrix is not read a second time.
+// exactly as they are stored, in fp64, and leaves it in gpart[chunk index][d] for `decode_sum_kernel` (or, with a
+// single chunk of workers, writes the decoded gradient itself): the coded matrix is not read a second time.
 template <typename CT, int S1, bool DEC>
 __global__ void __launch_bounds__(128)
 encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double *__restrict__ coef, int n,
                      long long d, int chunk, CT *__restrict__ coded, const double *__restrict__ avec,
-                     double *__restrict__ gpart) {
+                     double *__restrict__ gpart, float *__restrict__ grad) {
   pdl_sync();
   constexpr int W = S1 + kEncLook;
   __shared__ CT cs[NGC_MAX_N * S1];
@@ -590,10 +590,16 @@ encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double
     }
   }
   if constexpr (DEC) {
-    double *gp = gpart + (size_t)blockIdx.y * d + col;
+    if (gridDim.y == 1) {  // a single chunk of workers: this is the decoded gradient
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if (col + e < d) gp[e] = gacc[e];
+      for (int e = 0; e < 4; ++e)
+        if (col + e < d) grad[col + e] = (float)gacc[e];
+    } else {
+      double *gp = gpart + (size_t)blockIdx.y * d + col;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (col + e < d) gp[e] = gacc[e];
+    }
   }
 }
 
@@ -637,7 +643,8 @@ encode_simple_kernel(const RowSplit split, const float *__restrict__ ws, long lo
 }
 
 template <typename CT>
-using EncodeKernel = void (*)(const float *, long long, const double *, int, long long, int, CT *, const double *, double *);
+using EncodeKernel = void (*)(const float *, long long, const double *, int, long long, int, CT *, const double *, double *,
+                              float *);
 
 template <typename CT, bool DEC>
 EncodeKernel<CT> encode_window_for(int s1) {
@@ -687,9 +694,10 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
   const int chunk = (n + best_chunks - 1) / best_chunks;
   const dim3 grid((unsigned)col_blocks, (unsigned)((n + chunk - 1) / chunk));
   launch_k(kern, grid, 128, 0, stream, ws, ld_ws, coef, n, d, chunk, coded, fuse ? dec->a : nullptr,
-           fuse ? dec->gpart : nullptr);
+           fuse ? dec->gpart : nullptr, fuse ? dec->grad : nullptr);
   cudaError_t err = cudaGetLastError();
-  if (err != cudaSuccess || !fuse) return err;
+  if (fuse && dec->sum_launches) *dec->sum_launches = grid.y > 1 ? 1 : 0;
+  if (err != cudaSuccess || !fuse || grid.y == 1) return err;
   launch_k(decode_sum_kernel, (unsigned)((d + 255) / 256), 256, 0, stream, dec->gpart, (int)grid.y, d, dec->grad);
   return cudaGetLastError();
 }
