@@ -888,25 +888,35 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
 
 // [dW2; db2] of partition j = sum of the slots the head kernel's CTAs filled, in CTA order (reruns are
 // bit-identical).  blockIdx.y = partition.
-__global__ void head_reduce_kernel(const float *__restrict__ slots, int max_slots, int wstride, int tpp, int num_tiles,
-                                   int grid, float *__restrict__ G, size_t g_batch) {
-  pdl_sync();
-  const int j = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= wstride) return;
+struct HeadSlots {
+  const float *slots;  // [k][max_slots][wstride]; nullptr = nothing to add up
+  int max_slots, wstride, tpp, num_tiles, grid, k;
+  float *G;            // [dW2; db2] of partition j goes to G + j * g_batch
+  size_t g_batch;
+};
+
+// Element e of [dW2; db2] of partition j.
+__device__ __forceinline__ void head_reduce_one(const HeadSlots &h, int j, int e) {
   // CTAs of the head kernel whose tile range meets partition j
-  const int cfirst = (int)(((long long)(j * tpp + 1) * grid - 1) / num_tiles);
-  const int clast = (int)(((long long)((j + 1) * tpp) * grid - 1) / num_tiles);
-  const float *s0 = slots + (size_t)j * max_slots * wstride + e;
+  const int cfirst = (int)(((long long)(j * h.tpp + 1) * h.grid - 1) / h.num_tiles);
+  const int clast = (int)(((long long)((j + 1) * h.tpp) * h.grid - 1) / h.num_tiles);
+  const float *s0 = h.slots + (size_t)j * h.max_slots * h.wstride + e;
   const int nsl = clast - cfirst + 1;
   float acc = 0.f;
   for (int sb = 0; sb < nsl; sb += 8) {  // eight loads in flight, added in slot order
     float v[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = sb + i < nsl ? __ldg(s0 + (size_t)(sb + i) * wstride) : 0.f;
+    for (int i = 0; i < 8; ++i) v[i] = sb + i < nsl ? __ldg(s0 + (size_t)(sb + i) * h.wstride) : 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc += v[i];
   }
-  G[(size_t)j * g_batch + e] = acc;
+  h.G[(size_t)j * h.g_batch + e] = acc;
+}
+
+__global__ void head_reduce_kernel(const HeadSlots h) {
+  pdl_sync();
+  const int j = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e < h.wstride) head_reduce_one(h, j, e);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1285,6 +1295,7 @@ struct TnWideParams {
   size_t out_batch;
   int out_ld;
   int *status;
+  HeadSlots side;  // MLP: the head kernel's slots are added up by the epilogue warps while the first operands arrive
 };
 
 // Widths of the two instructions of pass `pass` (multiples of 32; w1 may be 0).
@@ -1394,6 +1405,11 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else {
     const int q = warp & 3, half = (warp - 2) >> 2;  // warps w and w + 4 share a quadrant and alternate 32-column chunks
+    if (p.side.slots) {
+      const long long total = (long long)p.side.k * p.side.wstride, nthr = (long long)gridDim.x * (kWideThreads - 64);
+      for (long long e = (long long)blockIdx.x * (kWideThreads - 64) + ((int)threadIdx.x - 64); e < total; e += nthr)
+        head_reduce_one(p.side, (int)(e / p.side.wstride), (int)(e % p.side.wstride));
+    }
     uint32_t aph = 0;
     for (int u = pair_id; u < p.num_units; u += n_pairs) {
       const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
@@ -1595,10 +1611,9 @@ size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
 }
 
 int mlp_launch_count(int hidden) {
-  // operand preparation, forward, head, dW1, encode; dW2 by a contraction of its own, or by the head kernel
-  // plus the sum over its slots
-  (void)hidden;
-  return 6;
+  // operand preparation, forward, head, dW1, encode; dW2 by a contraction of its own or by the head kernel plus a
+  // sum over its slots, which the wide backward kernel (hidden a multiple of 256) does on the side
+  return hidden % 256 == 0 ? 5 : 6;
 }
 
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
@@ -1681,6 +1696,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   }
   if (e != cudaSuccess) return e;
 
+  HeadSlots head_slots = {};
   if (head_tc) {
     CUtensorMap tmW2t, tmW2k, tmD1s;
     const uint64_t w2tdims[2] = {(uint64_t)hidden, 16}, w2kdims[2] = {64, (uint64_t)hidden};
@@ -1698,10 +1714,13 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     launch_k(mlp_head_tc_kernel, hgrid, kHeadTcThreads, head_tc_smem, stream, tmHa, tmW2t, tmW2k, tmD1s, hp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (fuse_w2) {
-      const int wstride = hidden * C + C;
-      launch_k(head_reduce_kernel, dim3((wstride + 255) / 256, k), 256, 0, stream, slots, max_slots, wstride, tpp, k * tpp, hgrid,
-                                                                            G + (size_t)d * hidden + hidden, lpad);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      head_slots.slots = slots; head_slots.max_slots = max_slots; head_slots.wstride = hidden * C + C;
+      head_slots.tpp = tpp; head_slots.num_tiles = k * tpp; head_slots.grid = hgrid; head_slots.k = k;
+      head_slots.G = G + (size_t)d * hidden + hidden; head_slots.g_batch = lpad;
+      if (!pair) {  // (the wide backward kernel below adds the slots up on the side)
+        launch_k(head_reduce_kernel, dim3((head_slots.wstride + 255) / 256, k), 256, 0, stream, head_slots);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      }
     }
   } else {
     const int cpad = (C + 3) / 4 * 4;
@@ -1735,6 +1754,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     wp.batch = k; wp.m_tiles = hidden / 256; wp.n_passes = (d + 1 + 511) / 512;
     wp.num_units = k * wp.m_tiles * wp.n_passes; wp.num_k = (rows + 63) / 64;
     wp.n_total = d + 1; wp.out = G; wp.out_batch = lpad; wp.out_ld = hidden; wp.status = status;
+    wp.side = head_slots;
     e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, tmD1, tmXb, wp, stream, kSmemWide);
   } else {
     launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmXb, tmD1, t);
