@@ -23,7 +23,10 @@ Pin status (what each part is checked against in the CPU test-suite):
                                    Carlo), the 0.95^8 ceiling of Section III,
                                    Observation 1 load bound, hand cases
   * partial gradients ............ finite differences of the loss, autograd,
-                                   normal equations
+                                   normal equations; the optional ReLU decision
+                                   of grad_mlp: identity with the default when
+                                   handed the default's own decision, a 2 x 2
+                                   case worked by hand, the all-ones mask
   * decoded gradient ............. equals the plain full-data gradient
 """
 from __future__ import annotations

@@ -12,6 +12,7 @@ from fractions import Fraction
 
 import numpy as np
 import pytest
+import scipy.special
 import scipy.stats
 import torch
 
@@ -236,6 +237,56 @@ def test_gradients_against_autograd(kind):
     assert np.allclose(g, th.grad.numpy(), rtol=1e-10, atol=1e-11)
 
 
+def test_mlp_relu_mask_argument():
+    # The optional ReLU decision: handing in the oracle's own decision (pre > 0) changes nothing, bit for bit ...
+    rng = np.random.default_rng(3)
+    rows, d, hidden, C = 17, 6, 5, 4
+    X = rng.normal(size=(rows, d))
+    y = rng.integers(0, C, rows)
+    theta = rng.normal(size=d * hidden + hidden + hidden * C + C)
+    W1 = theta[: d * hidden].reshape(d, hidden)
+    b1 = theta[d * hidden: d * hidden + hidden]
+    own = (X @ W1 + b1) > 0.0
+    g0 = orc.grad_mlp(X, y, theta, hidden, C)
+    assert np.array_equal(orc.grad_mlp(X, y, theta, hidden, C, relu_mask=own), g0)
+    assert np.array_equal(orc.grad_mlp(X, y, theta, hidden, C, relu_mask=own.astype(np.int8)), g0)
+    # ... an all-ones mask is the gradient of the network with the ReLU derivative replaced by 1 in the backward
+    # pass only: dW2, db2 (which never see the mask) stay, dW1 = X^T (delta2 W2^T) by hand
+    o = d * hidden + hidden
+    W2 = theta[o: o + hidden * C].reshape(hidden, C)
+    Z = np.maximum(X @ W1 + b1, 0) @ W2 + theta[o + hidden * C:]
+    P = np.exp(Z - scipy.special.logsumexp(Z, axis=1, keepdims=True))
+    P[np.arange(rows), y] -= 1.0
+    g1 = orc.grad_mlp(X, y, theta, hidden, C, relu_mask=np.ones((rows, hidden)))
+    assert np.allclose(g1[: d * hidden].reshape(d, hidden), X.T @ (P @ W2.T), rtol=1e-12, atol=1e-13)
+    assert np.allclose(g1[d * hidden: o], (P @ W2.T).sum(axis=0), rtol=1e-12, atol=1e-13)
+    assert np.array_equal(g1[o:], g0[o:])
+
+
+def test_mlp_relu_mask_hand_case_one_flipped_unit():
+    # 2 samples, 2 inputs, 2 hidden units, 2 classes, everything small enough to do by hand.
+    # W1 = I, b1 = 0, so pre = X; sample 0 = (1, -1): unit 1 is off; sample 1 = (2, 3): both on.
+    # W2 = [[1, 0], [0, 1]], b2 = 0.  Flipping the decision of (sample 0, unit 1) to "on" must add
+    # x_0 * (delta2_0 . W2[1]) to column 1 of dW1 and delta2_0 . W2[1] to db1[1], and touch nothing else.
+    X = np.array([[1.0, -1.0], [2.0, 3.0]])
+    y = np.array([0, 1])
+    theta = np.concatenate([np.eye(2).reshape(-1), np.zeros(2), np.eye(2).reshape(-1), np.zeros(2)])
+    base = orc.grad_mlp(X, y, theta, 2, 2)
+    mask = np.array([[1, 1], [1, 1]])                      # the oracle's own decision is [[1, 0], [1, 1]]
+    flipped = orc.grad_mlp(X, y, theta, 2, 2, relu_mask=mask)
+    # delta2 of sample 0 by hand: h = (1, 0), z = (1, 0), softmax = (e, 1) / (e + 1), label 0
+    p1 = 1.0 / (math.e + 1.0)
+    delta2_0 = np.array([-p1, p1])
+    extra = delta2_0[1]                                    # delta2_0 . W2[1] with W2 = I
+    diff = flipped - base
+    want = np.zeros_like(base)
+    want[0 * 2 + 1] = X[0, 0] * extra                      # dW1[0, 1]
+    want[1 * 2 + 1] = X[0, 1] * extra                      # dW1[1, 1]
+    want[4 + 1] = extra                                    # db1[1]
+    assert np.allclose(diff, want, rtol=0, atol=1e-15)
+    assert np.count_nonzero(diff) == 3
+
+
 # ------------------------------------------- decoded gradient = full gradient
 def _small_problem(kind, n, rows, d, hidden, C, seed):
     rng = np.random.default_rng(seed)
@@ -395,6 +446,52 @@ def test_erlang_reading_of_eq3():
             # identity in the proof of Corollary 1 (rho = 0)
             diff = latency.cdf_tasks(u, t, lam, 0.0, 0.0, 0.0) - latency.cdf_tasks(u + 1, t, lam, 0.0, 0.0, 0.0)
             assert abs(diff - math.exp(-lam * t) * (lam * t) ** u / math.factorial(u)) < 1e-12
+
+
+# ------------------------------------- the oracle's own task-time sampler (Section II-D)
+def test_oracle_trial_seed_is_the_published_stream():
+    # trial r of a run uses output r + 1 of the SplitMix64 stream seeded with (seed xor a fixed constant):
+    # with the seed chosen so that the xor gives 1234567, the published vector of the generator must come out
+    seed = 1234567 ^ 0xD1B54A32D192ED03
+    assert latency.trial_seed(seed, 0) == 6457827717110365317
+    assert latency.trial_seed(seed, 1) == 3203168211198807973
+    assert latency.trial_seed(seed, 4) == 16408922859458223821
+
+
+def test_oracle_sampler_follows_the_response_time_model():
+    # Section II-D: a task takes rho + Exp(lambda); a worker fails, with all its tasks, with probability p_e
+    n, tasks, rho, lam, pe = 4000, 5, 0.5, 2.0, 0.2
+    t = np.array(latency.sample_times(99, n, tasks, rho, lam, pe))
+    dead = np.isinf(t[:, 0])
+    assert all(np.isinf(t[i]).all() if dead[i] else np.isfinite(t[i]).all() for i in range(n))
+    assert abs(dead.mean() - pe) < 4 * math.sqrt(pe * (1 - pe) / n)
+    x = t[~dead].reshape(-1) - rho
+    assert x.min() > 0.0
+    m = x.size
+    assert abs(x.mean() - 1 / lam) < 5 / lam / math.sqrt(m)
+    assert abs(x.var() - 1 / lam ** 2) < 0.05 / lam ** 2
+    assert scipy.stats.kstest(x, "expon", args=(0, 1 / lam)).pvalue > 1e-3
+    # tasks of one worker and of different workers are not copies of each other
+    assert len(np.unique(x)) == m
+    # the first uniform of the stream, by hand: position 2 of seed 1234567 is 3203168211198807973
+    u = ((3203168211198807973 >> 11) + 0.5) / 2.0 ** 53
+    one = latency.sample_times(1234567, 1, 1, 0.25, 4.0, 0.0)[0][0]
+    assert abs(one - (0.25 - math.log(u) / 4.0)) < 1e-15
+
+
+@pytest.mark.parametrize("sigma", [0, 2])
+def test_lemma2_on_the_oracle_sampler(sigma):
+    # the same Monte Carlo as above, with the task times drawn by the oracle's SplitMix64 sampler
+    n, lam, rho, gamma, eps, pe, trials = 8, 0.5, 0.5, 0.3, 0.1, 0.05, 6000
+    T = np.full(trials, np.inf)
+    for r in range(trials):
+        t = np.array(latency.sample_times(latency.trial_seed(4242 + sigma, r), n, sigma + 1, rho, lam, pe))
+        out = orc.select(t, [sigma], gamma, eps)
+        if out is not None:
+            T[r] = out["latency"]
+    for t in (3.0, 5.0, 8.0, 12.0, 18.0):
+        want = latency.cdf_gc(t, n, sigma, lam, rho, gamma, eps, pe)
+        assert abs(np.mean(T <= t) - want) < 0.025, (t, np.mean(T <= t), want)
 
 
 # ----------------------------------------------------- stored oracle outputs
