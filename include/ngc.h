@@ -216,6 +216,8 @@ int ngc_sample_times(uint64_t seed, int n, int tasks, double shift, double rate,
  * Arguments are those of ngc_grad_encode; the plan is only read (its host tables), so a plan that
  * has never touched the GPU works.  status_dev may be NULL; if given, it points to one int32 in
  * device memory that is cleared by the call and set to 1 if a bounded device-side wait gave up.
+ * That word is the only place where such a timeout shows: without it the flag stays inside the
+ * array, and ngc_device_status, which reads the plan's own word, does not see this entry point.
  * Limit: n * slots * d * 4 bytes of partial gradients must fit in 8 MiB, where slots is the largest
  * number of CTAs that share one partition group (about 148 / n + 2 on a B200); larger problems are
  * refused with NGC_ERR_TOO_LARGE before anything is enqueued.
@@ -240,7 +242,7 @@ int ngc_grad_encode_static(const ngc_plan_t *plan, const ngc_model_t *model, con
  * device (trial r uses the ngc_sample_times stream of seed SplitMix64(seed ^ 0xD1B54A32D192ED03, r + 1)), run
  * through the stopping rule, and the latency (plan's gamma + eps + decode instant; +inf when no component ever
  * becomes decodable) and the chosen level (-1 when none) are written to latency_dev[trials] / level_dev[trials]
- * (device memory, either may be NULL).  Asynchronous on the stream.
+ * (device memory; one of the two may be NULL, not both).  Asynchronous on the stream.
  */
 double ngc_latency_cdf_gc(int n, int sigma, double t, double lambda, double rho, double gamma, double eps,
                           double p_fail);
@@ -261,8 +263,19 @@ int ngc_profile_read(ngc_plan_t *plan, double *ms_total_out, int64_t *launches_o
 /* Bytes of device workspace the plan currently holds. */
 size_t ngc_workspace_bytes(const ngc_plan_t *plan);
 /* Synchronises the device and returns NGC_OK or NGC_ERR_TIMEOUT / NGC_ERR_SINGULAR from the status
- * words the kernels of this plan wrote; *residual_out (may be NULL) gets the largest decode residual seen. */
+ * words the kernels of this plan wrote; *residual_out (may be NULL) gets the largest decode residual seen.
+ * A timeout is reported once: the call that returns NGC_ERR_TIMEOUT clears the word, so that the plan can
+ * be used, and judged, again. */
 int ngc_device_status(ngc_plan_t *plan, double *residual_out);
+/*
+ * Self-test of the failure path of the device-side waits (a property of the library; the paper has no
+ * counterpart).  Every wait of a kernel on a copy or on the tensor cores is bounded: after a cycle limit
+ * the kernel sets the plan's status word and returns instead of spinning.  This call enqueues one warp
+ * that waits at most limit_cycles (1 .. 2e9) SM cycles on a barrier that nothing will ever complete and
+ * then takes exactly that exit.  Afterwards ngc_device_status returns NGC_ERR_TIMEOUT (once), and the
+ * plan and the CUDA context remain usable.  Nothing faults or hangs.
+ */
+int ngc_selftest_wait_timeout(ngc_plan_t *plan, int64_t limit_cycles, void *cuda_stream);
 /* cudaError_t of the last failed runtime call on this plan (0 if none). */
 int ngc_last_cuda_error(const ngc_plan_t *plan);
 /* How many kernels of this library the plan has launched so far. */

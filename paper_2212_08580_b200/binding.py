@@ -80,6 +80,7 @@ def load_library() -> C.CDLL:
         "ngc_latency_mc": (i32, [vp, u64, i64, dbl, dbl, dbl, vp, vp, vp]),
         "ngc_gd_update": (i32, [vp, vp, i64, C.c_float, vp]),
         "ngc_sample_times": (i32, [u64, i32, i32, dbl, dbl, dbl, P(dbl)]),
+        "ngc_selftest_wait_timeout": (i32, [vp, i64, vp]),
         "ngc_profile_enable": (i32, [vp, i32]),
         "ngc_profile_read": (i32, [vp, P(dbl), P(i64)]),
         "ngc_workspace_bytes": (C.c_size_t, [vp]),
@@ -263,6 +264,14 @@ class Plan:
         res = C.c_double()
         self._check(self._lib.ngc_device_status(self._h, C.byref(res)), "ngc_device_status")
         return res.value
+
+    def device_status_code(self) -> int:
+        """Raw return value of ngc_device_status (0, NGC_ERR_TIMEOUT or NGC_ERR_SINGULAR)."""
+        return int(self._lib.ngc_device_status(self._h, None))
+
+    def selftest_wait_timeout(self, limit_cycles: int, stream: int = 0):
+        self._check(self._lib.ngc_selftest_wait_timeout(self._h, int(limit_cycles), stream),
+                    "ngc_selftest_wait_timeout")
 
     def profile_enable(self, on: bool):
         self._check(self._lib.ngc_profile_enable(self._h, int(on)), "ngc_profile_enable")

@@ -334,22 +334,15 @@ int ngc_decode(ngc_plan_t *p, int layer, const int32_t *S, int nS, const void *c
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
   NGC_CUDA(p, ngc::launch_decode(coded, coded_dtype, p->d_a, p->n, l, grad, stream));
-  if (p->ev_decoded) {
-    // tells the side stream of ngc_step that the vector has been read; an event recorded inside a stream
-    // capture could not be waited for by the eager steps that follow, and a captured step is in order anyway
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    NGC_CUDA(p, cudaStreamIsCapturing(stream, &cap));
-    if (cap == cudaStreamCaptureStatusNone)
-      NGC_CUDA(p, cudaEventRecord(static_cast<cudaEvent_t>(p->ev_decoded), stream));
-  }
   p->launches += 2;
   return NGC_OK;
 }
 
 // The decoding vector depends only on the responsive set, which is known before any gradient is:
 // ngc_step solves it on a stream of the plan's own, under the gradient kernels, and the decode on the
-// caller's stream waits for it.  The solve of one step in turn waits until the decode of the step
-// before has read the vector.  A capturing stream takes the plain in-order path.
+// caller's stream waits for it.  The solve in turn waits for everything the caller's stream held when the
+// step was entered (the decode of the step before reads the same vector).  A capturing stream takes the
+// plain in-order path.
 int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y,
              const double *task_times, void *coded, float *grad, ngc_step_info_t *info, void *cuda_stream) {
   if (!p || !info) return NGC_ERR_INVALID;
@@ -386,11 +379,12 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
     p->ev_solved = e1;
     NGC_CUDA(p, cudaEventCreateWithFlags(&e2, cudaEventDisableTiming));
     p->ev_decoded = e2;
-    // everything already queued on the caller's stream (an earlier ngc_decode, say) comes first
-    NGC_CUDA(p, cudaEventRecord(e2, stream));
   }
   cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);
   cudaEvent_t solved = static_cast<cudaEvent_t>(p->ev_solved), decoded = static_cast<cudaEvent_t>(p->ev_decoded);
+  // Everything already queued on the caller's stream comes before the solve overwrites the vector: the decode
+  // of the step before, but also a replayed graph whose captured steps recorded no event.
+  NGC_CUDA(p, cudaEventRecord(decoded, stream));
   NGC_CUDA(p, cudaStreamWaitEvent(side, decoded, 0));
   NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
   NGC_CUDA(p, cudaEventRecord(solved, side));
@@ -403,7 +397,6 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
     NGC_CUDA(p, ngc::launch_decode(coded, ngc_coded_dtype(p, m), p->d_a, p->n, ngc_num_params(m), grad, stream));
     p->launches += 1;
   }
-  NGC_CUDA(p, cudaEventRecord(decoded, stream));
   p->launches += 1;  // the solve
   return NGC_OK;
 }
@@ -437,7 +430,7 @@ int ngc_step_host(ngc_plan_t *p, const ngc_model_t *m, const float *theta, const
 int ngc_latency_mc(ngc_plan_t *p, uint64_t seed, int64_t trials, double rho, double lambda, double p_fail,
                    double *latency_dev, int32_t *level_dev, void *cuda_stream) {
   if (!p || trials < 1 || !(rho >= 0.0) || !(lambda > 0.0) || !(p_fail >= 0.0 && p_fail <= 1.0)) return NGC_ERR_INVALID;
-  if (!latency_dev || !level_dev) return NGC_ERR_INVALID;
+  if (!latency_dev && !level_dev) return NGC_ERR_INVALID;  // one of the two outputs may be left out
   NGC_CUDA(p, ngc::launch_latency_mc(*p, seed, trials, rho, lambda, p_fail, latency_dev, level_dev,
                                      static_cast<cudaStream_t>(cuda_stream)));
   p->launches += 1;
@@ -466,8 +459,20 @@ int ngc_device_status(ngc_plan_t *p, double *residual_out) {
   NGC_CUDA(p, cudaMemcpy(st, p->d_status, sizeof(st), cudaMemcpyDeviceToHost));
   NGC_CUDA(p, cudaMemcpy(&mr, p->d_maxres, sizeof(mr), cudaMemcpyDeviceToHost));
   if (residual_out) *residual_out = mr;
-  if (st[0] != 0) return NGC_ERR_TIMEOUT;
+  if (st[0] != 0) {  // reported once: the word is cleared so that later work on the plan is judged on its own
+    NGC_CUDA(p, cudaMemset(p->d_status, 0, sizeof(int)));
+    return NGC_ERR_TIMEOUT;
+  }
   if (!(mr <= kResidualLimit)) return NGC_ERR_SINGULAR;
+  return NGC_OK;
+}
+
+int ngc_selftest_wait_timeout(ngc_plan_t *p, int64_t limit_cycles, void *cuda_stream) {
+  if (!p || limit_cycles < 1 || limit_cycles > 2000000000ll) return NGC_ERR_INVALID;
+  const int rc = ensure_tables(p);
+  if (rc != NGC_OK) return rc;
+  NGC_CUDA(p, ngc::launch_wait_timeout(limit_cycles, p->d_status, static_cast<cudaStream_t>(cuda_stream)));
+  p->launches += 1;
   return NGC_OK;
 }
 

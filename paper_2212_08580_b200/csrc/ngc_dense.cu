@@ -203,10 +203,15 @@ __device__ __forceinline__ void convert_x_block(const float *__restrict__ X, __n
 //
 // Softmax residual R = softmax(z) - onehot(label), rounded to bf16: row max and row sum are exchanged through
 // `xch` ([2][2][128] floats) and a 64-thread named barrier per lane quadrant; one exponential per element.
+//
+// Failure handling of the forward epilogues: the 256 epilogue threads meet at named barriers, which have no
+// time limit, so a thread whose bounded wait gave up must not leave on its own.  It raises the shared abort
+// flag and walks on; everybody samples the flag between the tile's two block-wide barriers (`stop`), where
+// no thread can be writing it, and all leave together after the second one.
 template <typename Release>
 __device__ __forceinline__ void softmax_residual_row(uint32_t taddr, int ncol, int c_lo, int nch, int label,
                                                      __nv_bfloat16 *srow, float *xch, int rt, int half, int bar_id,
-                                                     Release release) {
+                                                     Release release, const volatile int *abort_flag, int &stop) {
   constexpr float kLog2e = 1.4426950408889634f;
   uint32_t r[128];
   tmem_ld_chunks<4>(taddr + c_lo * 32, nch, r);
@@ -242,6 +247,7 @@ __device__ __forceinline__ void softmax_residual_row(uint32_t taddr, int ncol, i
   const float inv = 1.f / (xch[256 + rt] + xch[256 + 128 + rt]);
   const int lm = label - c_lo * 32;  // position of the label among this thread's columns
   asm volatile("bar.sync 5, 256;" ::: "memory");  // the previous tile has left the staging buffer
+  stop = *abort_flag;
 #pragma unroll
   for (int g8 = 0; g8 < 16; ++g8) {  // 8 values = one 16-byte store
     uint32_t w[4];
@@ -260,12 +266,13 @@ __device__ __forceinline__ void softmax_residual_row(uint32_t taddr, int ncol, i
 // H = relu(z), rounded to bf16.
 template <typename Release>
 __device__ __forceinline__ void relu_row(uint32_t taddr, int ncol, int c_lo, int nch, __nv_bfloat16 *srow,
-                                         Release release) {
+                                         Release release, const volatile int *abort_flag, int &stop) {
   uint32_t r[128];
   tmem_ld_chunks<4>(taddr + c_lo * 32, nch, r);
   release();
   const int nmine = min(ncol - c_lo * 32, nch * 32);
   asm volatile("bar.sync 5, 256;" ::: "memory");  // the previous tile has left the staging buffer
+  stop = *abort_flag;
 #pragma unroll
   for (int g8 = 0; g8 < 16; ++g8) {
     uint32_t w[4];
@@ -359,8 +366,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     uint32_t aph = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
-      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
+      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; *s.abort_flag = 1; }
       tc_fence_after();
+      int stop = 0;
       const int rt = q * 32 + lane, row = rb * 128 + rt;
       const bool valid = row < p.rows;
       const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
@@ -375,13 +383,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         mbar_arrive(tempty_bar);
       };
       if (EPI == 0) {
-        softmax_residual_row(taddr, ncol, c_lo, nch, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release);
+        softmax_residual_row(taddr, ncol, c_lo, nch, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release,
+                             s.abort_flag, stop);
       } else {
-        relu_row(taddr, ncol, c_lo, nch, srow, release);
+        relu_row(taddr, ncol, c_lo, nch, srow, release, s.abort_flag, stop);
         if (valid && half == 0 && nt == 0 && p.ones_col >= 0)  // bf16 1.0 followed by zeros
           *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
       }
       asm volatile("bar.sync 5, 256;" ::: "memory");  // the tile is complete in shared memory
+      if (stop) break;  // (the same value in all 256 threads)
       store_staged_tile(s.stage, p.out + ((size_t)j * p.rows + rb * 128) * p.out_ld + nt * 256, p.out_ld,
                         p.rows - rb * 128, ncol, warp - 2, lane);
       buf ^= 1;
@@ -541,7 +551,6 @@ mlp_head_kernel(const __nv_bfloat16 *__restrict__ H, int hpad, int hidden, int C
 // ------------------------------------------------------------------------------------------------
 constexpr int kHeadEpiThreads = 512;  // 16 epilogue warps: four per tensor-memory quadrant
 constexpr int kHeadTcThreads = 96 + kHeadEpiThreads;  // + two producer warps and the MMA warp
-__device__ __forceinline__ void head_epi_sync() { asm volatile("bar.sync 6, %0;" ::"n"(kHeadEpiThreads) : "memory"); }
 
 struct HeadTcParams {
   int hidden, C, rows, tiles_per_part, num_tiles;  // a tile = 128 rows of one partition
@@ -627,6 +636,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[17]);
   float *b2s = reinterpret_cast<float *>(&bars[18]);          // 16 floats
   float *dbx = reinterpret_cast<float *>(&bars[26]);          // [4 quadrants][16]: bias-gradient partial sums
+  const uint32_t epi_bar = smem_u32(&bars[58]);               // meeting point of the epilogue threads (bounded, unlike bar.sync)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -641,6 +651,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
     mbar_init(d_full, 1);
     mbar_init(d_empty, kHeadEpiThreads);
     mbar_init(w_full, 1);
+    mbar_init(epi_bar, kHeadEpiThreads);
     mbar_fence_init();
   }
   if (threadIdx.x < 16) b2s[threadIdx.x] = (int)threadIdx.x < p.C ? p.b2[threadIdx.x] : 0.f;
@@ -746,7 +757,15 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
     const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;  // row r inside a swizzled tile
     const uint32_t rx = (uint32_t)(r & 7);
     const int wstride = p.hidden * p.C + p.C;
-    uint32_t ph = 0, dph = 0;
+    uint32_t ph = 0, dph = 0, eph = 0;
+    // all epilogue threads meet: arrive, then a bounded wait for the others (a thread that gave up elsewhere
+    // never arrives, and the rest then give up here instead of waiting for ever)
+    auto epi_sync = [&]() -> bool {
+      mbar_arrive(epi_bar);
+      const bool ok = mbar_wait(epi_bar, eph);
+      eph ^= 1u;
+      return ok;
+    };
     float db2_acc = 0.f;  // lane c of a part-0 warp: sum of delta2[., c] over the warp's rows
     for (int tile = t_begin; tile < t_end; ++tile) {
       const int j = tile / tpp, rb = tile % tpp;
@@ -873,10 +892,10 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
           if (lane < 16) dbx[q * 16 + lane] = db2_acc;
           db2_acc = 0.f;
         }
-        head_epi_sync();
+        if (!epi_sync()) { failed = true; break; }
         if (tid_epi < p.C)
           dst[(size_t)p.hidden * p.C + tid_epi] = (dbx[tid_epi] + dbx[16 + tid_epi]) + (dbx[32 + tid_epi] + dbx[48 + tid_epi]);
-        head_epi_sync();  // dbx is free again
+        if (!epi_sync()) { failed = true; break; }  // dbx is free again
       }
     }
   }
@@ -1032,6 +1051,7 @@ struct PairSmem {
   unsigned char *tiles;
   uint32_t full[kPairStages], empty[kPairStages], tfull[2], tempty[2];
   uint32_t *tmem_slot;
+  volatile int *abort_flag;
   float *xch;
   __nv_bfloat16 *stage;
 };
@@ -1050,6 +1070,7 @@ __device__ __forceinline__ PairSmem carve_pair(unsigned char *raw) {
   s.tempty[0] = smem_u32(&bars[2 * kPairStages + 2]);
   s.tempty[1] = smem_u32(&bars[2 * kPairStages + 3]);
   s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kPairStages + 4]);
+  s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
   s.xch = reinterpret_cast<float *>(s.tiles + kPairStages * kPairStageBytes + 256);
   s.stage = reinterpret_cast<__nv_bfloat16 *>(s.tiles + kPairStages * kPairStageBytes + 256 + kXchBytes);
   return s;
@@ -1065,6 +1086,7 @@ __device__ __forceinline__ uint32_t pair_prologue(const PairSmem &s, int warp, i
     mbar_init(s.tfull[1], 1);
     mbar_init(s.tempty[0], 2 * epi_threads);
     mbar_init(s.tempty[1], 2 * epi_threads);
+    *s.abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(s.tmem_slot), kTmemCols);
@@ -1146,8 +1168,9 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     uint32_t aph = 0;
     for (int tile = pair_id; tile < p.num_tiles; tile += n_pairs) {
       const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
-      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
+      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; *s.abort_flag = 1; }
       tc_fence_after();
+      int stop = 0;
       const int rt = q * 32 + lane, row = rb * 256 + (int)rank * 128 + rt;
       const bool valid = row < p.rows;
       const size_t grow = (size_t)j * p.rows + (valid ? row : 0);
@@ -1160,13 +1183,15 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         mbar_arrive_cluster(tempty_bar);
       };
       if (EPI == 0) {
-        softmax_residual_row(taddr, 256, c_lo, 4, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release);
+        softmax_residual_row(taddr, 256, c_lo, 4, valid ? p.y[grow] : -1, srow, s.xch, rt, half, 1 + q, release,
+                             s.abort_flag, stop);
       } else {
-        relu_row(taddr, 256, c_lo, 4, srow, release);
+        relu_row(taddr, 256, c_lo, 4, srow, release, s.abort_flag, stop);
         if (valid && half == 0 && nt == 0 && p.ones_col >= 0)
           *reinterpret_cast<uint4 *>(p.out + grow * p.out_ld + p.ones_col) = make_uint4(0x00003f80u, 0u, 0u, 0u);
       }
       asm volatile("bar.sync 5, 256;" ::: "memory");
+      if (stop) break;  // (the same value in all 256 threads)
       store_staged_tile(s.stage, p.out + ((size_t)j * p.rows + rb * 256 + (int)rank * 128) * p.out_ld + nt * 256,
                         p.out_ld, p.rows - rb * 256 - (int)rank * 128, 256, warp - 2, lane);
       buf ^= 1;

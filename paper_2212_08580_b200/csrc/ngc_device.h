@@ -87,6 +87,9 @@ cudaError_t launch_latency_mc(const ngc_plan_s &plan, uint64_t seed, long long t
 // theta <- theta - step * grad (Eq. 1).
 cudaError_t launch_gd_update(float *theta, const float *grad, long long l, float step, cudaStream_t stream);
 
+// One warp waits at most `limit_cycles` SM cycles on a barrier nobody arrives on, then sets *status to 1.
+cudaError_t launch_wait_timeout(long long limit_cycles, int *status, cudaStream_t stream);
+
 int device_sm_count();
 
 }  // namespace ngc

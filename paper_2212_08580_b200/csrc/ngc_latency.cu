@@ -64,8 +64,8 @@ __global__ void __launch_bounds__(128) latency_mc_kernel(const McParams p) {
     }
     if (D < best) { best = D; best_l = l; }
   }
-  p.latency[trial] = best_l < 0 ? INFINITY : p.gamma + p.eps + best;
-  p.level[trial] = best_l;
+  if (p.latency) p.latency[trial] = best_l < 0 ? INFINITY : p.gamma + p.eps + best;
+  if (p.level) p.level[trial] = best_l;
 }
 
 }  // namespace

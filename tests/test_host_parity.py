@@ -106,6 +106,12 @@ def test_argument_errors():
     assert p.coded_dtype(ngc.Model.make("mlp", "f32", 10, 784, 10, 512)) == ngc.NGC_F32
     p.set_coded_dtype(ngc.NGC_F32)
     assert p.coded_dtype(ngc.Model.make("lsq", "f32", 10, 32)) == ngc.NGC_F32
+    # Monte Carlo of the stopping rule: one of the two outputs may be left out, not both (checked before any launch)
+    lib = ngc.load_library()
+    assert lib.ngc_latency_mc(p._h, 1, 16, 0.5, 0.5, 0.05, None, None, None) == -1
+    assert lib.ngc_latency_mc(p._h, 1, 0, 0.5, 0.5, 0.05, None, None, None) == -1
+    assert lib.ngc_selftest_wait_timeout(p._h, 0, None) == -1
+    assert lib.ngc_selftest_wait_timeout(None, 1000, None) == -1
 
 
 def test_sample_times_model():

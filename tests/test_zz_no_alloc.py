@@ -12,7 +12,8 @@ import torch
 
 import ngc_inputs
 import paper_2212_08580_b200 as ngc
-from tests._util import coded_torch_dtype, model_of, rel_l2
+from oracle import ngc_oracle as orc
+from tests._util import coded_torch_dtype, model_of, oracle_G, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -33,16 +34,27 @@ def test_static_variant_matches_allocating_entry_point_twice_in_a_row():
         static_plan = ngc.Plan(w.n, w.levels, seed=w.seed)             # never allocates on the device
         cdt = ref_plan.coded_dtype(m)
         status = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+        G = oracle_G(w, X, y, theta)                                   # the CPU oracle, from the same bits
+        B = orc.plan(w.n, list(w.levels), w.seed)["B"]
         for layer in range(len(w.levels)):
             want = torch.empty((w.n, w.d), dtype=coded_torch_dtype(cdt), device="cuda")
             got = torch.full_like(want, float("nan"))
             ref_plan.grad_encode(m, theta, X, y, layer, want)
+            static_plan.grad_encode_static(m, theta, X, y, layer, got, status)   # (first call: loads the module)
+            torch.cuda.synchronize()
+            # nothing is allocated or freed on the device: the driver's free-memory figure does not move across
+            # further calls (torch's caching allocator is left alone in between)
+            free0, _ = torch.cuda.mem_get_info()
             static_plan.grad_encode_static(m, theta, X, y, layer, got, status)
             torch.cuda.synchronize()
+            free1, _ = torch.cuda.mem_get_info()
+            assert free1 == free0
             assert int(status.item()) == 0
             assert static_plan.workspace_bytes() == 0
+            want_oracle = orc.encode(B[layer], G)
             for i in range(w.n):
                 assert rel_l2(got[i].cpu().numpy(), want[i].cpu().numpy()) < TOL
+                assert rel_l2(got[i].cpu().numpy(), want_oracle[i]) < TOL
         # status pointer is optional
         got2 = torch.full_like(got, float("nan"))
         static_plan.grad_encode_static(m, theta, X, y, len(w.levels) - 1, got2)
