@@ -112,6 +112,41 @@ def make_data(w: Workload, device="cpu"):
     raise ValueError(w.kind)
 
 
+def make_data_batched(w: Workload, device="cpu"):
+    """Same distributions as `make_data`, all partitions drawn by one call per tensor (a handful of
+    launches on a GPU).  For small cases only: the whole data matrix exists in fp32 for a moment.  The
+    values differ from `make_data`'s for the same seed (the generator is consumed in another order)."""
+    dev = torch.device(device)
+    g = _gen(w.seed, dev)
+    xdt = torch.bfloat16 if w.x_dtype == "bf16" else torch.float32
+    shape = (w.n, w.rows, w.d)
+    if w.kind in ("lsq", "logistic"):
+        std = 1.0 if w.unit_x else 1.0 / math.sqrt(w.d)
+        theta_star = torch.randn(w.d, generator=g, device=dev)
+        theta = torch.randn(w.d, generator=g, device=dev)
+        X = (torch.randn(shape, generator=g, device=dev) * std).to(xdt)
+        z = X.float() @ theta_star
+        if w.kind == "lsq":
+            y = z + 0.1 * torch.randn((w.n, w.rows), generator=g, device=dev)
+        else:
+            y = (torch.rand((w.n, w.rows), generator=g, device=dev) < torch.sigmoid(z)).float()
+        return X, y, theta
+    y = torch.randint(0, w.n_classes, (w.n, w.rows), generator=g, device=dev, dtype=torch.int32)
+    if w.kind == "softmax":
+        X = (torch.randn(shape, generator=g, device=dev) / math.sqrt(w.d)).to(xdt)
+        return X, y, 0.1 * torch.randn(w.d * w.n_classes, generator=g, device=dev)
+    if w.kind == "mlp":
+        X = torch.rand(shape, generator=g, device=dev).to(xdt)
+        theta = torch.zeros(w.n_params, device=dev)
+        o = w.d * w.hidden
+        theta[:o] = torch.randn(o, generator=g, device=dev) * math.sqrt(2.0 / w.d)
+        o2 = o + w.hidden
+        theta[o2:o2 + w.hidden * w.n_classes] = (torch.randn(w.hidden * w.n_classes, generator=g, device=dev)
+                                                 * math.sqrt(2.0 / w.hidden))
+        return X, y, theta
+    raise ValueError(w.kind)
+
+
 def sample_times(n: int, n_tasks: int, seed: int, shift=1.0, rate=1.0, p_fail=0.0) -> np.ndarray:
     """Per-task durations [n, n_tasks]: shift + Exp(rate) i.i.d.; a worker fails
     (all its tasks +inf) independently with probability p_fail."""

@@ -58,7 +58,7 @@ def build(verbose: bool = False) -> str:
             if log:
                 print(log)
     if _newer(objs, LIB):
-        cmd = [NVCC, "-shared", "-o", LIB, *objs, "-cudart", "static", "-lcuda" if False else "-ldl"]
+        cmd = [NVCC, "-shared", "-o", LIB, *objs, "-cudart", "static", "-ldl"]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"link failed: {' '.join(cmd)}\n{r.stdout}\n{r.stderr}")
