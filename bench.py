@@ -4,9 +4,11 @@
 One "step" = one full iteration for a fresh seeded straggler pattern: stopping rule, fused
 partial gradients + encode for the chosen component code, decoding-vector solve, decode.
 
-    python bench.py --gpus 1 --steps 200 --warmup 20            # CUDA library
+    python bench.py --gpus 1 --steps 200 --warmup 20            # CUDA library, headline workload + the other three
+    python bench.py --workload mlp30 --only                     # one workload, nothing else
     python bench.py --impl reference --steps 2 --warmup 1       # the CPU oracle, on the host cores
     torchrun --nproc-per-node N ... bench.py --gpus N ...       # N independent replicas (weak scaling)
+    torchrun --nproc-per-node N ... bench.py --gpus N --sharded # ONE problem, partitions sharded over the ranks
 
 Prints ONE JSON line on rank 0.
 """
@@ -19,6 +21,7 @@ import statistics
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 import numpy as np
@@ -31,8 +34,15 @@ import ngc_inputs  # noqa: E402
 
 METRIC = "decoded NGC gradients/sec"
 UNIT = "gradients/s"
-DEFAULT_WORKLOAD = "logistic20"
+DEFAULT_WORKLOAD = "lsq100"          # the largest single-GPU configuration (6.57 GB per step)
+SIDE_WORKLOADS = ("logistic20", "softmax50", "mlp30", "lsq100")
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per full-size launch of the timed kernel (dense workloads: summed
+# over the gradient kernels the events bracket), from the ncu captures summarised under profiles/; None = the
+# kernels have changed since the counters were taken.
+TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000, "softmax50": None, "mlp30": None}
 
 
 # ----------------------------------------------------------------------------- small helpers
@@ -93,24 +103,20 @@ def algorithmic_flops(w: ngc_inputs.Workload) -> int:
     return w.n * w.rows * (4 * w.d * w.hidden + 6 * w.hidden * w.n_classes)
 
 
-# dram__bytes_read + dram__bytes_write per full-size launch of the timed kernel (the dense workloads: summed over the
-# gradient kernels the events bracket), from the ncu captures summarised under profiles/ (None = not captured for
-# the kernels as they stand).
-TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000,
-                 "softmax50": 1_075_000_000, "mlp30": 643_000_000}
-FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
-
-
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             return json.load(f), "measured"
-    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops_sustained": FALLBACK_BF16_TFLOPS_SUSTAINED}, "fallback"
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while a timed region runs (read-only queries).
+
+    NVML in a thread of this process every few milliseconds (the timed regions last tens of milliseconds);
+    `nvidia-smi -lms` as a fallback.  Samples taken while the GPU reports itself idle are kept apart, so that
+    `sm_mhz` is the median UNDER LOAD."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -119,8 +125,36 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.thread = None
+        self.stop_flag = False
+        self.samples = []          # (sm_mhz, reasons bit mask, power W)
+        self.max_mhz = None
+        self.nvml = None
+
+    def _loop(self, handle):
+        nv = self.nvml
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(handle)
+                watts = nv.nvmlDeviceGetPowerUsage(handle) / 1000.0
+                self.samples.append((float(mhz), int(reasons), watts))
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            handle = nv.nvmlDeviceGetHandleByIndex(self.gpu)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+            self.nvml = nv
+            self.thread = threading.Thread(target=self._loop, args=(handle,), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
@@ -132,6 +166,25 @@ class ClockSampler:
 
     def stop(self) -> dict:
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            nv = self.nvml
+            idle_bit = nv.nvmlClocksThrottleReasonGpuIdle
+            names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                     "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                     "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                     "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+            busy = [s for s in self.samples if not (s[1] & idle_bit)]
+            use = busy if busy else self.samples
+            if use:
+                out["sm_mhz"] = statistics.median(s[0] for s in use)
+                out["sm_max_mhz"] = self.max_mhz
+                out["samples"] = len(self.samples)
+                out["samples_under_load"] = len(busy)
+                out["power_w_max"] = max(s[2] for s in use)
+                out["reasons"] = sorted(k for k, bit in names.items() if any(s[1] & bit for s in use))
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -173,13 +226,11 @@ def oracle_threads() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_step_seconds(w, X, y, theta, times, sample_rows: int):
-    """Times the oracle as it stands on a bounded sample of one step.
-
-    The partial gradients are computed on the first `sample_rows` rows of the workload (whole partitions
-    first, then a row prefix of the next one) and that time is scaled to all n * rows rows; selection,
-    encode, decoding vector and decode are timed in full (on the sampled gradients tiled to n rows).
-    """
+def oracle_reduced_step(w, X, y, theta, times, rows_r: int):
+    """One step of the oracle, as it stands, on a reduced copy of the workload: every partition cut to its first
+    `rows_r` rows (X, y: host tensors [n, >= rows_r, ...]).  Selection, the n partial gradients, encode, decoding
+    vector and decode all run.  Returns (seconds scaled to the full workload, seconds spent, decoded gradient):
+    the partial gradients' time is scaled by rows / rows_r, the rest is taken as it is."""
     from oracle import ngc_oracle as orc
     levels = list(w.levels)
     pl = orc.plan(w.n, levels, w.seed)
@@ -188,28 +239,34 @@ def oracle_step_seconds(w, X, y, theta, times, sample_rows: int):
     t_sel = time.perf_counter() - t0
     th = theta.double().numpy()
     t0 = time.perf_counter()
-    Gs, left, j = [], sample_rows, 0
-    while left > 0:
-        r = min(left, w.rows)
-        yj = y[j, :r].double().numpy() if y.dtype.is_floating_point else y[j, :r].numpy()
-        Gs.append(orc.partial_gradient(w.kind, X[j, :r].double().numpy(), yj, th, w.hidden, w.n_classes))
-        left -= r
-        j += 1
-    t_grad = (time.perf_counter() - t0) * (w.n * w.rows / sample_rows)
-    G = np.stack([Gs[j % len(Gs)] for j in range(w.n)])
+    Gs = []
+    for j in range(w.n):
+        yj = y[j, :rows_r].double().numpy() if y.dtype.is_floating_point else y[j, :rows_r].numpy()
+        Gs.append(orc.partial_gradient(w.kind, X[j, :rows_r].double().numpy(), yj, th, w.hidden, w.n_classes))
+    t_grad = time.perf_counter() - t0
+    G = np.stack(Gs)
     t0 = time.perf_counter()
     B = pl["B"][sel["level"]]
     coded = orc.encode(B, G)
     a = orc.decode_vector(B, sel["S"])
-    orc.decode(a, coded)
+    g = orc.decode(a, coded)
     t_rest = time.perf_counter() - t0
-    return t_sel + t_grad + t_rest
+    spent = t_sel + t_grad + t_rest
+    return t_sel + t_grad * (w.rows / rows_r) + t_rest, spent, g
 
 
-def sample_description(w, sample_rows, secs=None):
-    s = (f"partial gradients on the first {sample_rows} of {w.n * w.rows} rows, time scaled "
-         f"x{w.n * w.rows / sample_rows:.4g}; selection, encode, decoding vector and decode in full")
-    return s + (f" ({secs:.2f} s/step)" if secs is not None else "")
+def rows_within_budget(w, X, y, theta, times, budget_s: float) -> int:
+    """Rows per partition the oracle can take in about `budget_s` seconds, extrapolated from a probe on the
+    first rows of every partition (X, y hold at least that many)."""
+    probe = max(1, min(w.rows, int(X.shape[1])))
+    _, spent, _ = oracle_reduced_step(w, X, y, theta, times, probe)
+    return int(max(1, min(w.rows, probe * budget_s / max(spent, 1e-6))))
+
+
+def sample_description(w, rows_r, secs=None):
+    s = (f"one oracle step on a reduced copy: all {w.n} partitions cut to their first {rows_r} of {w.rows} rows; "
+         f"partial-gradient time scaled x{w.rows / rows_r:.4g}, selection, encode, decoding vector and decode as timed")
+    return s + (f" ({secs:.2f} s/step at full size)" if secs is not None else "")
 
 
 def run_reference(args):
@@ -217,26 +274,18 @@ def run_reference(args):
     rank, _, world = env_rank()
     if rank != 0:
         return
-    from dataclasses import replace
-
     from oracle import ngc_oracle as orc
     w = ngc_inputs.WORKLOADS[args.workload]
-    budget = args.cpu_budget_s / max(1, args.steps + args.warmup)      # seconds of oracle work per step
-    # one partition first: how long does a row take?
-    X, y, theta = ngc_inputs.make_data(replace(w, n=1), "cpu")
-    probe_rows = min(w.rows, 256)
+    budget = args.cpu_budget_s / max(1, args.steps + args.warmup + 1)      # seconds of oracle work per step
     pats = [ngc_inputs.pattern_times(w, it) for it in range(args.warmup + args.steps + 64)]
     pats = [t for t in pats if orc.select(t, list(w.levels), 0.0, 0.0) is not None]
-    t0 = time.perf_counter()
-    oracle_step_seconds(w, X, y, theta, pats[0], probe_rows)
-    per_row = max((time.perf_counter() - t0) / probe_rows, 1e-9)
-    sample_rows = int(min(w.n * w.rows, max(16, budget / per_row)))
-    parts = -(-sample_rows // w.rows)
-    if parts > 1:
-        X, y, theta = ngc_inputs.make_data(replace(w, n=parts), "cpu")
+    # a first guess from a small copy, then the copy the budget allows
+    X, y, theta = ngc_inputs.make_data(ngc_inputs.shrink(w, rows=max(1, min(w.rows, 32))), "cpu")
+    rows_r = rows_within_budget(w, X, y, theta, pats[0], budget)
+    X, y, theta = ngc_inputs.make_data(ngc_inputs.shrink(w, rows=rows_r), "cpu")
     for i in range(args.warmup):
-        oracle_step_seconds(w, X, y, theta, pats[i], sample_rows)
-    secs = [oracle_step_seconds(w, X, y, theta, pats[args.warmup + i], sample_rows) for i in range(args.steps)]
+        oracle_reduced_step(w, X, y, theta, pats[i], rows_r)
+    secs = [oracle_reduced_step(w, X, y, theta, pats[args.warmup + i], rows_r)[0] for i in range(args.steps)]
     total = sum(secs)
     value = args.steps / total
     line = {
@@ -246,7 +295,7 @@ def run_reference(args):
         "config": {"workload": w.name, "n_workers": w.n, "levels": list(w.levels), "kind": w.kind,
                    "rows_per_partition": w.rows, "d": w.d, "x_dtype": w.x_dtype},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                         "sample": sample_description(w, sample_rows)},
+                         "sample": sample_description(w, rows_r)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -254,9 +303,175 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+class Problem:
+    """One workload resident on the device, with its plan and output buffers."""
+
+    def __init__(self, w, dev, prepare: bool):
+        import torch
+        import paper_2212_08580_b200 as ngc
+        self.ngc, self.torch = ngc, torch
+        self.w, self.dev = w, dev
+        self.X, self.y, self.theta = ngc_inputs.make_data(w, dev)
+        self.m = ngc.Model.make(w.kind, w.x_dtype, w.rows, w.d, w.n_classes, w.hidden)
+        self.plan = ngc.Plan(w.n, w.levels, seed=w.seed)
+        self.cdt = self.plan.coded_dtype(self.m)
+        self.l = w.n_params
+        self.coded = torch.empty((w.n, self.l), dtype=torch.float64 if self.cdt == ngc.NGC_F64 else torch.float32,
+                                 device=dev)
+        self.grad = torch.empty(self.l, dtype=torch.float32, device=dev)
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.prep_ms = None
+        if prepare:
+            # The data matrix is assigned to the workers once, before training (Section II-C): whatever the
+            # library derives from it alone (a bf16 copy for the tensor cores) is made once, outside the steps.
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.plan.prepare_data(self.m, self.X, self.stream)
+            e1.record()
+            torch.cuda.synchronize()
+            self.prep_ms = e0.elapsed_time(e1)
+
+    def decodable(self, t):
+        try:
+            self.plan.select(t)
+            return True
+        except self.ngc.NgcError:
+            return False
+
+    def step(self, t):
+        return self.plan.step(self.m, self.theta, self.X, self.y, t, self.coded, self.grad, self.stream)
+
+
+def roofline_of(w, cdt_is_f64, kern_ms, kern_n, peaks, which, traffic):
+    kern_avg_ms = kern_ms / max(kern_n, 1)
+    if w.kind in ("lsq", "logistic"):
+        alg = algorithmic_bytes(w, 8 if cdt_is_f64 else 4)
+        achieved = alg / (kern_avg_ms * 1e-3) / 1e9 if kern_n else None
+        return {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": traffic,
+                "kernel": "gemv_pair_kernel", "kernel_ms": kern_avg_ms, "algorithmic_bytes": alg,
+                "peak_source": f"of {which}"}
+    flops = algorithmic_flops(w)
+    peak = peaks.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS_SUSTAINED)
+    achieved = flops / (kern_avg_ms * 1e-3) / 1e12 if kern_n else None
+    return {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+            "kernel": "gradient kernels of one call (operand layouts, forward, head, backward contractions)",
+            "kernel_ms": kern_avg_ms, "algorithmic_flops": flops, "peak_source": f"of {which} (sustained bf16)"}
+
+
+def timed_steps(pb, pats, steps):
+    """`steps` steps queued back to back between two events on the launching stream (the product's own launch
+    sequence: no event sits between its kernels).  Returns (total ms, levels chosen)."""
+    torch = pb.torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    levels = []
+    e0.record()
+    for i in range(steps):
+        levels.append(pb.step(pats[i]).layer)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1), levels
+
+
+def per_step_median_ms(pb, pats, steps):
+    """Median over `steps` steps, each between its own pair of events (queued without host synchronisation)."""
+    torch = pb.torch
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
+        pb.step(pats[i % len(pats)])
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+
+
+def kernel_bracket(pb, pats, steps):
+    """A pass of its own with the library's event brackets around the gradient kernels of every call."""
+    pb.plan.profile_read()
+    pb.plan.profile_enable(True)
+    for i in range(steps):
+        pb.step(pats[i % len(pats)])
+    pb.torch.cuda.synchronize()
+    ms, n = pb.plan.profile_read()
+    pb.plan.profile_enable(False)
+    return ms, n
+
+
+def host_queue_us(pb, pats, steps):
+    """Host time of one ngc_step call (argument checks, stopping rule, launches), steps queued without waiting."""
+    pb.torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(steps):
+        pb.step(pats[i % len(pats)])
+    dt = time.perf_counter() - t0
+    pb.torch.cuda.synchronize()
+    return 1e6 * dt / steps
+
+
+def cpu_baseline_and_parity(pb, pats, budget_s):
+    """The oracle, as it stands, timed on the host cores on a reduced copy of the workload; the library then runs
+    the same reduced problem, which gives the parity figure of this very run."""
+    torch, w = pb.torch, pb.w
+    Xh = pb.X[:, : min(w.rows, 32)].cpu()
+    yh = pb.y[:, : min(w.rows, 32)].cpu()
+    th = pb.theta.cpu()
+    rows_r = rows_within_budget(w, Xh, yh, th, pats[0], budget_s)
+    Xr = pb.X[:, :rows_r].contiguous()
+    yr = pb.y[:, :rows_r].contiguous()
+    secs, _, g_oracle = oracle_reduced_step(w, Xr.cpu(), yr.cpu(), th, pats[0], rows_r)
+    mr = pb.ngc.Model.make(w.kind, w.x_dtype, rows_r, w.d, w.n_classes, w.hidden)
+    plan_r = pb.ngc.Plan(w.n, w.levels, seed=w.seed)
+    pb.grad.zero_()
+    plan_r.step(mr, pb.theta, Xr, yr, pats[0], pb.coded, pb.grad, pb.stream)
+    torch.cuda.synchronize()
+    got = pb.grad.double().cpu().numpy()
+    err = float(np.linalg.norm(got - g_oracle) / max(np.linalg.norm(g_oracle), 1e-300))
+    plan_r.close()
+    base = {"value": 1.0 / secs, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": sample_description(w, rows_r, secs)}
+    parity = {"rel_l2_vs_oracle": err, "tolerance": 1e-5 if w.kind in ("lsq", "logistic") else 1e-2,
+              "on": f"the reduced copy of the cpu_baseline leg ({rows_r} rows per partition)"}
+    return base, parity
+
+
+def measure_side_workload(name, dev, peaks, which, smi_index, args):
+    """Median step time, kernel-bracket roofline, clocks and parity of one workload (N = 1 only)."""
+    import torch
+    w = ngc_inputs.WORKLOADS[name]
+    pb = Problem(w, dev, prepare=not args.no_prepare)
+    steps, warm = max(100, args.side_steps), 20
+    pats, skipped = decodable_patterns(w, w.levels, steps, pb.decodable)
+    for i in range(warm):
+        pb.step(pats[i])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(smi_index)
+    sampler.start()
+    time.sleep(0.05)
+    total_ms, levels = timed_steps(pb, pats, steps)
+    med = per_step_median_ms(pb, pats, steps)
+    kern_ms, kern_n = kernel_bracket(pb, pats, min(steps, 50))
+    clocks = sampler.stop()
+    host_us = host_queue_us(pb, pats, steps)
+    out = {"ms_per_step": med, "ms_per_step_mean_of_queued": total_ms / steps, "steps": steps, "warmup": warm,
+           "gradients_per_s": 1e3 / med,
+           "roofline": roofline_of(w, pb.cdt == pb.ngc.NGC_F64, kern_ms, kern_n, peaks, which, TRAFFIC_BYTES.get(name)),
+           "clocks": clocks, "host_us_per_step_call": host_us, "prep_ms_once": pb.prep_ms,
+           "undecodable_skipped": skipped,
+           "levels_chosen": {str(k): levels.count(k) for k in sorted(set(levels))},
+           "decode_residual_max": pb.plan.device_status()}
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"], out["parity"] = cpu_baseline_and_parity(pb, pats, args.side_cpu_s)
+    pb.plan.close()
+    del pb
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
-    import paper_2212_08580_b200 as ngc
+    import paper_2212_08580_b200 as ngc  # noqa: F401  (fails loudly when the CUDA library is missing)
 
     rank, local_rank, world = env_rank()
     if world != args.gpus:
@@ -268,33 +483,18 @@ def run_cuda(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+    if args.sharded:
+        from paper_2212_08580_b200 import sharded
+        return sharded.bench_sharded(args, rank, local_rank, world, dev)
 
     w = replica_workload(ngc_inputs.WORKLOADS[args.workload], rank)
     if args.rows:                      # reduced case for profiler captures; never the reported workload
         w = ngc_inputs.shrink(w, rows=args.rows)
-    X, y, theta = ngc_inputs.make_data(w, dev)
-    m = ngc.Model.make(w.kind, w.x_dtype, w.rows, w.d, w.n_classes, w.hidden)
-    plan = ngc.Plan(w.n, w.levels, seed=w.seed)
-    cdt = plan.coded_dtype(m)
-    l = w.n_params
-    coded = torch.empty((w.n, l), dtype=torch.float64 if cdt == ngc.NGC_F64 else torch.float32, device=dev)
-    grad = torch.empty(l, dtype=torch.float32, device=dev)
-
-    def decodable(t):
-        try:
-            plan.select(t)
-            return True
-        except ngc.NgcError:
-            return False
-
-    pats, skipped = decodable_patterns(w, w.levels, args.warmup + args.steps, decodable)
-    stream = torch.cuda.current_stream().cuda_stream
-
+    pb = Problem(w, dev, prepare=not args.no_prepare)
+    pats, skipped = decodable_patterns(w, w.levels, args.warmup + max(args.steps, args.median_steps), pb.decodable)
     for i in range(args.warmup):
-        plan.step(m, theta, X, y, pats[i], coded, grad, stream)
+        pb.step(pats[i])
     torch.cuda.synchronize()
-    plan.profile_read()
-    plan.profile_enable(True)
     try:
         smi_index = int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
     except (KeyError, ValueError, IndexError):
@@ -302,31 +502,28 @@ def run_cuda(args):
     sampler = ClockSampler(smi_index)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    launches0 = plan.launch_count()
+        time.sleep(0.05)
+    launches0 = pb.plan.launch_count()
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    levels_used = []
-    e0.record()
-    for i in range(args.steps):
-        info = plan.step(m, theta, X, y, pats[args.warmup + i], coded, grad, stream)
-        levels_used.append(info.layer)
-    e1.record()
-    torch.cuda.synchronize()
+    # ---- the timed region: exactly `steps` steps, the product's launch sequence, events on the launching stream
+    ms_local, levels_used = timed_steps(pb, pats[args.warmup:], args.steps)
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    ms_total = rank_max(e0.elapsed_time(e1), world, dev)
-    launches = plan.launch_count() - launches0
-    kern_ms, kern_n = plan.profile_read()
-    plan.profile_enable(False)
+    ms_total = rank_max(ms_local, world, dev)
+    launches = pb.plan.launch_count() - launches0
+    # ---- separate passes: per-step median, then the event brackets around the gradient kernels
+    median_ms = per_step_median_ms(pb, pats[args.warmup:], args.median_steps) if args.median_steps else None
+    kern_ms, kern_n = kernel_bracket(pb, pats[args.warmup:], min(max(args.steps, 20), 100))
     clocks = sampler.stop() if rank == 0 else {}
-    residual = plan.device_status()
+    host_us = host_queue_us(pb, pats[args.warmup:], min(max(args.steps, 20), 200))
+    residual = pb.plan.device_status()
 
     # ---- end to end through the host-buffer entry point: pinned host inputs copied every step
+    X, y, theta, l = pb.X, pb.y, pb.theta, pb.l
     e2e_steps = min(args.steps, args.e2e_steps)
     h2d = X.numel() * X.element_size() + y.numel() * y.element_size() + theta.numel() * 4
     d2h = l * 4
@@ -335,38 +532,22 @@ def run_cuda(args):
         Xh, yh, thh = X.cpu().pin_memory(), y.cpu().pin_memory(), theta.cpu().pin_memory()
         gh = torch.empty(l, dtype=torch.float32).pin_memory()
         for i in range(2):
-            plan.step_host(m, thh, Xh, yh, pats[i], gh)
+            pb.plan.step_host(pb.m, thh, Xh, yh, pats[i], gh)
         if world > 1:
             import torch.distributed as dist
             dist.barrier()
         t0 = time.perf_counter()
         for i in range(e2e_steps):
-            plan.step_host(m, thh, Xh, yh, pats[args.warmup + i], gh)
+            pb.plan.step_host(pb.m, thh, Xh, yh, pats[args.warmup + i], gh)
         torch.cuda.synchronize()
         e2e_s = rank_max(time.perf_counter() - t0, world, dev)
         e2e = {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+        del Xh, yh, thh, gh
 
-    # ---- roofline of the dominant kernel(s) (the fused gradient kernels that ngc_profile brackets)
     peaks, which = measured_peaks()
-    cbytes = 8 if cdt == ngc.NGC_F64 else 4
-    kern_avg_ms = kern_ms / max(kern_n, 1)
     traffic = TRAFFIC_BYTES.get(w.name) if not args.rows else None
-    if w.kind in ("lsq", "logistic"):
-        alg = algorithmic_bytes(w, cbytes)
-        achieved = alg / (kern_avg_ms * 1e-3) / 1e9 if kern_n else None
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": traffic,
-                    "kernel": "gemv_pair_kernel", "kernel_ms": kern_avg_ms, "algorithmic_bytes": alg,
-                    "peak_source": f"of {which}"}
-    else:
-        flops = algorithmic_flops(w)
-        peak = peaks.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS_SUSTAINED)
-        achieved = flops / (kern_avg_ms * 1e-3) / 1e12 if kern_n else None
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                    "kernel": "forward + backward contraction kernels", "kernel_ms": kern_avg_ms,
-                    "algorithmic_flops": flops, "peak_source": f"of {which} (sustained bf16)"}
+    roofline = roofline_of(w, pb.cdt == pb.ngc.NGC_F64, kern_ms, kern_n, peaks, which, traffic)
 
     line = {
         "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -375,25 +556,41 @@ def run_cuda(args):
         "dtype": "f32" if w.kind in ("lsq", "logistic") else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "n_workers": w.n, "levels": list(w.levels), "kind": w.kind,
                    "rows_per_partition": w.rows, "d": w.d, "x_dtype": w.x_dtype,
-                   "coded_dtype": "f64" if cdt == ngc.NGC_F64 else "f32",
+                   "coded_dtype": "f64" if pb.cdt == pb.ngc.NGC_F64 else "f32",
                    "l2": "inputs larger than L2 (data matrix %.2f GB per step)" % (h2d / 1e9),
                    "patterns": "fresh seeded pattern per step", "undecodable_skipped": skipped,
                    "levels_chosen": {str(k): levels_used.count(k) for k in sorted(set(levels_used))},
-                   "replicas": "independent per GPU, no data-path collective"},
+                   "replicas": "independent per GPU, no data-path collective",
+                   "data_prepared_once": (None if pb.prep_ms is None else
+                                          "ngc_prepare_data before the steps (Section II-C: the data is assigned once); "
+                                          "for the MLP it holds a bf16 copy of the data matrix, for the other models "
+                                          "nothing; its time is prep_ms_once, outside the timed region")},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(rank_sum(launches, world, dev)),
         "roofline": roofline,
+        "ms_per_step_median": median_ms,
+        "host_us_per_step_call": host_us,
+        "prep_ms_once": pb.prep_ms,
         "decode_residual_max": residual,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and e2e is not None:
-        t0 = time.perf_counter()
-        oracle_step_seconds(w, Xh, yh, thh, pats[0], min(w.rows, 256))
-        per_row = max((time.perf_counter() - t0) / min(w.rows, 256), 1e-9)
-        sample_rows = int(min(w.n * w.rows, max(16, args.cpu_budget_s / 6 / per_row)))
-        secs = oracle_step_seconds(w, Xh, yh, thh, pats[0], sample_rows)
-        line["cpu_baseline"] = {"value": 1.0 / secs, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                                "sample": sample_description(w, sample_rows, secs)}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"], line["parity"] = cpu_baseline_and_parity(pb, pats, args.cpu_budget_s / 8)
+    if rank == 0 and world == 1 and not args.only and not args.rows:
+        # the other configurations, each measured the same way (median of >= 100 steps), so that one run of the
+        # default command leaves a record for all four
+        pb.plan.close()
+        del pb, X, y, theta
+        torch.cuda.empty_cache()
+        side = {}
+        for name in SIDE_WORKLOADS:
+            if name == w.name:
+                side[name] = {"ms_per_step": median_ms if median_ms is not None else ms_total / args.steps,
+                              "roofline": roofline, "clocks": clocks, "parity": line.get("parity"),
+                              "see": "top level of this line"}
+                continue
+            side[name] = measure_side_workload(name, dev, peaks, which, smi_index, args)
+        line["workloads"] = side
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -408,7 +605,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(ngc_inputs.WORKLOADS))
+    ap.add_argument("--only", action="store_true", help="measure the named workload only (no `workloads` object)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one problem sharded over the ranks (strong scaling) instead of independent replicas")
+    ap.add_argument("--no-prepare", action="store_true", help="do not call ngc_prepare_data before the steps")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--median-steps", type=int, default=100, help="steps of the per-step median pass (0 = skip)")
+    ap.add_argument("--side-steps", type=int, default=100)
+    ap.add_argument("--side-cpu-s", type=float, default=4.0,
+                    help="seconds of CPU-oracle work per side workload")
     ap.add_argument("--cpu-budget-s", type=float, default=120.0,
                     help="seconds of CPU-oracle work the reference arm may spend in total")
     ap.add_argument("--no-cpu-baseline", action="store_true")

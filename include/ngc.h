@@ -145,6 +145,18 @@ int ngc_grad_encode(ngc_plan_t *plan, const ngc_model_t *model, const void *thet
                     const void *y_dev, int layer, void *coded_dev, void *cuda_stream);
 
 /*
+ * Once-only preparation of the data matrix (Section II-C: the main node assigns the row blocks to the
+ * workers at the beginning of training; they do not change from iteration to iteration).  Whatever the
+ * library derives from the data alone is made here instead of in every ngc_grad_encode / ngc_step:
+ * for NGC_MLP a bf16 copy of X_dev with a column of ones (the tensor cores' operand; device memory owned
+ * by the plan, counted by ngc_workspace_bytes); nothing for the other models, whose kernels read X_dev as
+ * it is.  Later calls that pass this same X_dev with the same model shape use the copy; calls with any
+ * other pointer convert per call as before.  Call it again when the contents of X_dev change; X_dev =
+ * NULL drops the copy.  Asynchronous on the stream (an allocation on first use aside).
+ */
+int ngc_prepare_data(ngc_plan_t *plan, const ngc_model_t *model, const void *X_dev, void *cuda_stream);
+
+/*
  * Decoding vectors (Definition 1: a row of A with support in S and a B = 1), computed
  * on the device by a batched fp64 solve.  S lists responsive workers in increasing
  * order, nS >= n - s_l; if nS is larger, the n - s_l smallest indices are used, which

@@ -68,6 +68,7 @@ def load_library() -> C.CDLL:
         "ngc_set_coded_dtype": (i32, [vp, i32]),
         "ngc_coded_dtype": (i32, [vp, P(Model)]),
         "ngc_select": (i32, [vp, P(dbl), P(StepInfo)]),
+        "ngc_prepare_data": (i32, [vp, P(Model), vp, vp]),
         "ngc_grad_encode": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp]),
         "ngc_grad_encode_static": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp, vp]),
         "ngc_decode_vector": (i32, [vp, i32, P(C.c_int32), i32, P(dbl)]),
@@ -210,6 +211,11 @@ class Plan:
         return info
 
     # ---- device path
+    def prepare_data(self, model: Model, X, stream: int = 0):
+        """ngc_prepare_data: what the library derives from the data matrix alone, made once (X=None drops it)."""
+        self._check(self._lib.ngc_prepare_data(self._h, C.byref(model), _addr(X) if X is not None else None, stream),
+                    "ngc_prepare_data")
+
     def grad_encode(self, model: Model, theta, X, y, layer: int, coded, stream: int = 0):
         self._check(self._lib.ngc_grad_encode(self._h, C.byref(model), _addr(theta), _addr(X), _addr(y), layer,
                                               _addr(coded), stream), "ngc_grad_encode")

@@ -135,7 +135,7 @@ extern "C" {
 
 void ngc_plan_destroy(ngc_plan_t *p) {
   if (!p) return;
-  if (p->tables_on_device || p->ws || p->st_X) {
+  if (p->tables_on_device || p->ws || p->st_X || p->dense_state) {
     cudaDeviceSynchronize();
     for (auto &lv : p->lv) {
       cudaFree(lv.d_coef);
@@ -155,6 +155,7 @@ void ngc_plan_destroy(ngc_plan_t *p) {
     cudaFree(p->st_coded);
     cudaFree(p->st_grad);
   }
+  ngc::dense_state_free(static_cast<ngc::DenseState *>(p->dense_state));
   for (void *e : p->ev) cudaEventDestroy(static_cast<cudaEvent_t>(e));
   if (p->ev_solved) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_solved));
   if (p->ev_decoded) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_decoded));
@@ -249,7 +250,8 @@ int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, con
     if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     NGC_CUDA(p, ngc::launch_softmax_grad(p->k, m->rows_per_partition, m->d, m->n_classes, X, static_cast<const int *>(y),
                                          static_cast<const float *>(theta), static_cast<unsigned char *>(p->ws), &G,
-                                         p->d_status, sms, stream));
+                                         p->d_status, sms, stream,
+                                         reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
     if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     // G is [n][q][l]: group g of q consecutive partitions, one scratch slot per partition
     ngc::RowSplit split;
@@ -273,7 +275,8 @@ int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, con
     if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     NGC_CUDA(p, ngc::launch_mlp_grad(p->k, m->rows_per_partition, m->d, h, C, static_cast<const float *>(X),
                                      static_cast<const int *>(y), static_cast<const float *>(theta),
-                                     static_cast<unsigned char *>(p->ws), &G, &ldG, p->d_status, sms, stream));
+                                     static_cast<unsigned char *>(p->ws), &G, &ldG, p->d_status, sms, stream,
+                                     reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
     if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
     ngc::RowSplit split;
     split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
@@ -287,6 +290,18 @@ int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, con
 }  // namespace
 
 extern "C" {
+
+int ngc_prepare_data(ngc_plan_t *p, const ngc_model_t *m, const void *X, void *cuda_stream) {
+  if (!p) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  if (m->kind != NGC_MLP) return NGC_OK;  // the other models read the data matrix as it is
+  if (m->x_dtype != NGC_F32 || m->d % 8 != 0 || (X && !aligned16(X))) return NGC_ERR_INVALID;
+  NGC_CUDA(p, ngc::prepare_mlp_data(reinterpret_cast<ngc::DenseState **>(&p->dense_state), p->k, m->rows_per_partition,
+                                    m->d, static_cast<const float *>(X), static_cast<cudaStream_t>(cuda_stream)));
+  if (X) p->launches += 1;
+  return NGC_OK;
+}
 
 int ngc_decode_vectors(ngc_plan_t *p, int layer, const int32_t *S, int nS, int batch, double *a_out,
                        double *resid_out) {
@@ -445,7 +460,8 @@ int ngc_gd_update(float *theta, const float *grad, int64_t l, float step, void *
 
 size_t ngc_workspace_bytes(const ngc_plan_t *p) {
   if (!p) return 0;
-  return p->ws_bytes + p->gpart_bytes + p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes +
+  return p->ws_bytes + p->gpart_bytes + ngc::dense_state_bytes(static_cast<const ngc::DenseState *>(p->dense_state)) +
+         p->st_X_bytes + p->st_y_bytes + p->st_theta_bytes + p->st_coded_bytes +
          p->st_grad_bytes;
 }
 

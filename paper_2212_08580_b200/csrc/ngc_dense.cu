@@ -11,6 +11,8 @@
 // Warp roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (+ tensor-memory owner), warps 2-5
 // epilogue (one accumulator row per thread).  Two 256-column accumulators let the epilogue of one
 // tile overlap the contraction of the next.
+#include <new>
+
 #include "ngc_device.h"
 #include "ngc_pdl.cuh"
 #include "ngc_tc.cuh"
@@ -1464,11 +1466,24 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   pair_teardown(warp, tmem_base, failed, p.status);
 }
 
+// The opt-in shared-memory size of a kernel is set once per device, not on every launch.
+template <typename Kern>
+cudaError_t ensure_smem_attr(Kern kern, int smem_bytes) {
+  static int done_bytes[64] = {};  // per device: the size already set for this kernel (one static per instantiation)
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && done_bytes[dev] >= smem_bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) done_bytes[dev] = smem_bytes;
+  return e;
+}
+
 // Launch on clusters of two CTAs.
 template <typename Kern, typename Params>
 cudaError_t launch_pair(Kern kern, int threads, int pair_tiles, int sms, const CUtensorMap &m0, const CUtensorMap &m1,
                         const Params &p, cudaStream_t stream, int smem_bytes = kSmemPair) {
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  cudaError_t e = ensure_smem_attr(kern, smem_bytes);
   if (e != cudaSuccess) return e;
   int pairs = sms / 2;
   if (pair_tiles < pairs) pairs = pair_tiles;
@@ -1528,7 +1543,63 @@ bool make_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+// Largest number of CTAs of the head kernel whose contiguous tile ranges touch one partition.
+int head_max_slots(int k, int tpp, int grid) {
+  int worst = 1;
+  for (int j = 0; j < k; ++j) {
+    // first and last CTA whose range [begin(c), begin(c + 1)) meets the tiles [j tpp, (j + 1) tpp) of partition j
+    const int cfirst = (int)(((long long)(j * tpp + 1) * grid - 1) / ((long long)k * tpp));
+    const int clast = (int)(((long long)((j + 1) * tpp) * grid - 1) / ((long long)k * tpp));
+    if (clast - cfirst + 1 > worst) worst = clast - cfirst + 1;
+  }
+  return worst;
+}
+
+int head_grid(int k, int rows, int sms) {
+  const int tiles = k * ((rows + 127) / 128);
+  return tiles < sms ? tiles : (sms > 0 ? sms : 1);
+}
+
 }  // namespace
+
+// What the dense launchers keep between calls, per plan: the tensor maps and derived sizes of the last
+// softmax and MLP problem (encoding 5-9 maps and walking the head kernel's tile ranges on every call is host
+// time on the critical path of a caller that synchronises per step), and the data prepared once.
+struct DenseState {
+  struct {
+    bool valid = false;
+    int k = 0, rows = 0, d = 0, C = 0;
+    const void *X = nullptr, *scratch = nullptr;
+    CUtensorMap tmXa, tmXb, tmW, tmWh, tmR;
+  } sm;
+  struct {
+    bool valid = false;
+    int k = 0, rows = 0, d = 0, hidden = 0, C = 0, sms = 0;
+    const void *Xb = nullptr, *scratch = nullptr;
+    int max_slots = 0;
+    CUtensorMap tmXa, tmXb, tmW, tmWh, tmH, tmHa, tmD1, tmD1s, tmD2, tmW2t, tmW2k;
+  } mlp;
+  // bf16 copy [X 1] of an MLP's data matrix made by prepare_mlp_data (owned here)
+  __nv_bfloat16 *Xb_prep = nullptr;
+  size_t Xb_prep_bytes = 0;
+  const void *prep_src = nullptr;
+  int prep_k = 0, prep_rows = 0, prep_d = 0;
+};
+
+void dense_state_free(DenseState *st) {
+  if (!st) return;
+  if (st->Xb_prep) cudaFree(st->Xb_prep);
+  delete st;
+}
+
+size_t dense_state_bytes(const DenseState *st) { return st ? st->Xb_prep_bytes : 0; }
+
+static DenseState *state_of(DenseState **slot) {
+  if (!*slot) *slot = new (std::nothrow) DenseState();
+  return *slot;
+}
 
 size_t softmax_scratch_bytes(int k, int rows, int d, int C) {
   const size_t wt = ((size_t)C * d * 2 + 255) / 256 * 256;
@@ -1538,8 +1609,11 @@ size_t softmax_scratch_bytes(int k, int rows, int d, int C) {
 }
 
 cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, const int *y, const float *W,
-                                unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream) {
+                                unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream,
+                                DenseState **state) {
   if (C % 16 != 0 || C < 16 || C > 256 || d % 8 != 0 || d < 8) return cudaErrorInvalidValue;
+  DenseState *st = state_of(state);
+  if (!st) return cudaErrorMemoryAllocation;
   const size_t wt_bytes = ((size_t)C * d * 2 + 255) / 256 * 256;
   const size_t r_bytes = ((size_t)k * rows * C * 2 + 255) / 256 * 256;
   __nv_bfloat16 *Wt = reinterpret_cast<__nv_bfloat16 *>(scratch);
@@ -1547,25 +1621,26 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   float *G = reinterpret_cast<float *>(scratch + wt_bytes + r_bytes);
   *G_out = G;
 
-  CUtensorMap tmXa, tmXb, tmW, tmR;
-  const uint64_t xdims[3] = {(uint64_t)d, (uint64_t)rows, (uint64_t)k};
-  const uint32_t xbox_a[3] = {64, 128, 1}, xbox_b[3] = {64, 64, 1};
-  const uint64_t wdims[2] = {(uint64_t)d, (uint64_t)C};
-  const uint32_t wbox[2] = {64, 256};
-  const uint64_t rdims[3] = {(uint64_t)C, (uint64_t)rows, (uint64_t)k};
-  const uint32_t rbox[3] = {64, 64, 1};
-  if (!make_map(&tmXa, X, 3, xdims, xbox_a) || !make_map(&tmXb, X, 3, xdims, xbox_b) ||
-      !make_map(&tmW, Wt, 2, wdims, wbox) || !make_map(&tmR, R, 3, rdims, rbox))
-    return cudaErrorInvalidValue;
+  auto &c = st->sm;
+  if (!(c.valid && c.k == k && c.rows == rows && c.d == d && c.C == C && c.X == X && c.scratch == scratch)) {
+    c.valid = false;
+    const uint64_t xdims[3] = {(uint64_t)d, (uint64_t)rows, (uint64_t)k};
+    const uint32_t xbox_a[3] = {64, 128, 1}, xbox_b[3] = {64, 64, 1};
+    const uint64_t wdims[2] = {(uint64_t)d, (uint64_t)C};
+    const uint32_t wbox[2] = {64, 256}, wbox_h[2] = {64, 128};  // whole tile / half of the class rows per CTA of a pair
+    const uint64_t rdims[3] = {(uint64_t)C, (uint64_t)rows, (uint64_t)k};
+    const uint32_t rbox[3] = {64, 64, 1};
+    if (!make_map(&c.tmXa, X, 3, xdims, xbox_a) || !make_map(&c.tmXb, X, 3, xdims, xbox_b) ||
+        !make_map(&c.tmW, Wt, 2, wdims, wbox) || !make_map(&c.tmWh, Wt, 2, wdims, wbox_h) ||
+        !make_map(&c.tmR, R, 3, rdims, rbox))
+      return cudaErrorInvalidValue;
+    c.k = k; c.rows = rows; c.d = d; c.C = C; c.X = X; c.scratch = scratch;
+    c.valid = true;
+  }
 
   dim3 tg((C + 31) / 32, (d + 31) / 32);
   launch_k(transpose_to_bf16_kernel, tg, 256, 0, stream, W, nullptr, Wt, d, C, d);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-
-  e = cudaFuncSetAttribute(fwd_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFwd);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
 
   const bool pair = (C == 256) && sms >= 2;
@@ -1574,16 +1649,14 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   p.num_k = (d + 63) / 64;
   p.y = y; p.out = R; p.out_ld = C; p.ones_col = -1; p.status = status;
   if (pair) {
-    CUtensorMap tmWh;  // half of the class rows per CTA
-    const uint32_t wbox_h[2] = {64, 128};
-    if (!make_map(&tmWh, Wt, 2, wdims, wbox_h)) return cudaErrorInvalidValue;
     p.row_blocks = (rows + 255) / 256;
     p.num_tiles = k * p.row_blocks;
-    e = launch_pair(fwd_pair_kernel<0>, kFwdThreads, p.num_tiles, sms, tmXa, tmWh, p, stream);
+    e = launch_pair(fwd_pair_kernel<0>, kFwdThreads, p.num_tiles, sms, c.tmXa, c.tmWh, p, stream);
   } else {
+    if ((e = ensure_smem_attr(fwd_kernel<0>, kSmemFwd)) != cudaSuccess) return e;
     p.row_blocks = (rows + 127) / 128;
     p.num_tiles = k * p.row_blocks;
-    launch_k(fwd_kernel<0>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, tmXa, tmW, p);
+    launch_k(fwd_kernel<0>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, c.tmXa, c.tmW, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
@@ -1597,32 +1670,12 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   t.status = status;
   if (pair) {
     t.m_tiles = (d + 255) / 256; t.num_tiles = k * t.m_tiles;
-    return launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, tmXb, tmR, t, stream);
+    return launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, c.tmXb, c.tmR, t, stream);
   }
+  if ((e = ensure_smem_attr(tn_gemm_kernel, kSmemTc)) != cudaSuccess) return e;
   t.m_tiles = (d + 127) / 128; t.num_tiles = k * t.m_tiles;
-  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmXb, tmR, t);
+  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, c.tmXb, c.tmR, t);
   return cudaGetLastError();
-}
-
-namespace {
-inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
-}  // namespace
-
-// Largest number of CTAs of the head kernel whose contiguous tile ranges touch one partition.
-static int head_max_slots(int k, int tpp, int grid) {
-  int worst = 1;
-  for (int j = 0; j < k; ++j) {
-    int cnt = 0;
-    for (int c = 0; c < grid; ++c)
-      if (head_tile_begin(c + 1, k * tpp, grid) > j * tpp && head_tile_begin(c, k * tpp, grid) < (j + 1) * tpp) ++cnt;
-    if (cnt > worst) worst = cnt;
-  }
-  return worst;
-}
-
-static int head_grid(int k, int rows, int sms) {
-  const int tiles = k * ((rows + 127) / 128);
-  return tiles < sms ? tiles : (sms > 0 ? sms : 1);
 }
 
 size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C) {
@@ -1641,12 +1694,59 @@ int mlp_launch_count(int hidden) {
   return hidden % 256 == 0 ? 5 : 6;
 }
 
+// bf16 copy [X 1] of the data matrix of an MLP, made once: the data is assigned to the workers before
+// training starts (Section II-C) and does not change from iteration to iteration, so the conversion the
+// tensor cores need (fp32 -> bf16, plus the column of ones that carries the bias) is no part of a step.
+// X == nullptr drops the copy.
+cudaError_t prepare_mlp_data(DenseState **state, int k, int rows, int d, const float *X, cudaStream_t stream) {
+  DenseState *st = state_of(state);
+  if (!st) return cudaErrorMemoryAllocation;
+  st->prep_src = nullptr;
+  st->mlp.valid = false;
+  if (!X) {
+    if (st->Xb_prep) {
+      cudaError_t e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return e;
+      cudaFree(st->Xb_prep);
+      st->Xb_prep = nullptr;
+      st->Xb_prep_bytes = 0;
+    }
+    return cudaSuccess;
+  }
+  if (d % 8 != 0 || k < 1 || rows < 1) return cudaErrorInvalidValue;
+  const int dpad = (d + 1 + 7) / 8 * 8;
+  const size_t kr = (size_t)k * rows, bytes = up256(kr * dpad * 2);
+  if (bytes > st->Xb_prep_bytes) {
+    if (st->Xb_prep) {
+      cudaError_t e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return e;
+      cudaFree(st->Xb_prep);
+      st->Xb_prep = nullptr;
+      st->Xb_prep_bytes = 0;
+    }
+    cudaError_t e = cudaMalloc(&st->Xb_prep, bytes);
+    if (e != cudaSuccess) return e;
+    st->Xb_prep_bytes = bytes;
+  }
+  MlpPrepParams pp = {};
+  pp.X = X; pp.Xb = st->Xb_prep; pp.rows_total = (long long)kr; pp.d = d; pp.dpad = dpad;
+  pp.tr_bx = 1; pp.tr_blocks = 0; pp.w2_blocks = 0;
+  const long long groups = (long long)kr * (dpad / 8);
+  launch_k(mlp_prep_kernel, (unsigned)((groups + 255) / 256), 256, 0, stream, pp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  st->prep_src = X; st->prep_k = k; st->prep_rows = rows; st->prep_d = d;
+  return cudaSuccess;
+}
+
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
                             unsigned char *scratch, float **G_out, long long *G_ld, int *status, int sms,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, DenseState **state) {
   if (d % 8 != 0 || hidden % 16 != 0 || hidden < 16 || hidden > 512 || (hidden > 256 && hidden % 256 != 0) || C < 1 ||
       C > 16)
     return cudaErrorInvalidValue;
+  DenseState *st = state_of(state);
+  if (!st) return cudaErrorMemoryAllocation;
   const int dpad = (d + 1 + 7) / 8 * 8, hpad = (hidden + 1 + 7) / 8 * 8;
   const size_t l = (size_t)d * hidden + hidden + (size_t)hidden * C + C, lpad = (l + 3) / 4 * 4;
   const size_t kr = (size_t)k * rows;
@@ -1658,48 +1758,63 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   __nv_bfloat16 *D2 = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256(kr * 64 * 2);
   __nv_bfloat16 *W2t = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)16 * hidden * 2);
   __nv_bfloat16 *W2k = reinterpret_cast<__nv_bfloat16 *>(ptr); ptr += up256((size_t)hidden * 64 * 2);
+  // the copy made by prepare_mlp_data for this very data matrix replaces the per-call conversion
+  const bool prepared = st->Xb_prep && st->prep_src == X && st->prep_k == k && st->prep_rows == rows && st->prep_d == d;
+  if (prepared) Xb = st->Xb_prep;
   const int tpp = (rows + 127) / 128, hgrid = head_grid(k, rows, sms);
-  const int max_slots = head_max_slots(k, tpp, head_grid(k, rows, device_sm_count()));
-  if (head_max_slots(k, tpp, hgrid) > max_slots) return cudaErrorInvalidValue;
-  float *slots = reinterpret_cast<float *>(ptr); ptr += up256((size_t)k * max_slots * ((size_t)hidden * C + C) * 4);
-  float *G = reinterpret_cast<float *>(ptr);
-  *G_out = G;
-  *G_ld = (long long)lpad;
-  const float *W1 = theta, *b1 = theta + (size_t)d * hidden, *W2 = b1 + hidden, *b2 = W2 + (size_t)hidden * C;
-
-  CUtensorMap tmXa, tmXb, tmW, tmH, tmD1, tmD2;
-  const uint64_t xdims[3] = {(uint64_t)dpad, (uint64_t)rows, (uint64_t)k};
-  const uint32_t box_a[3] = {64, 128, 1}, box_b[3] = {64, 64, 1};
-  const uint64_t wdims[2] = {(uint64_t)dpad, (uint64_t)hidden};
-  const uint32_t wbox[2] = {64, 256};
-  const uint64_t hdims[3] = {(uint64_t)hpad, (uint64_t)rows, (uint64_t)k};
-  const uint64_t d1dims[3] = {(uint64_t)hidden, (uint64_t)rows, (uint64_t)k};
-  const uint64_t d2dims[3] = {64, (uint64_t)rows, (uint64_t)k};
-  CUtensorMap tmHa;  // h in 128-row boxes (head), tmH in 64-row boxes (backward operand)
-  if (!make_map(&tmXa, Xb, 3, xdims, box_a) || !make_map(&tmXb, Xb, 3, xdims, box_b) ||
-      !make_map(&tmW, W1t, 2, wdims, wbox) || !make_map(&tmH, H, 3, hdims, box_b) || !make_map(&tmHa, H, 3, hdims, box_a) ||
-      !make_map(&tmD1, D1, 3, d1dims, box_b) || !make_map(&tmD2, D2, 3, d2dims, box_b))
-    return cudaErrorInvalidValue;
 
   const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
   const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 512 + 1024;
   const bool head_tc = hidden % 64 == 0 && head_tc_smem <= 232448;
   const bool fuse_w2 = head_tc && hidden % 128 == 0;  // the head forms [dW2; db2] itself: no column of ones behind h
 
+  auto &c = st->mlp;
+  if (!(c.valid && c.k == k && c.rows == rows && c.d == d && c.hidden == hidden && c.C == C && c.sms == sms &&
+        c.Xb == Xb && c.scratch == scratch)) {
+    c.valid = false;
+    // scratch was sized with the slot count of a grid on every SM of the device
+    c.max_slots = head_max_slots(k, tpp, head_grid(k, rows, device_sm_count()));
+    if (head_max_slots(k, tpp, hgrid) > c.max_slots) return cudaErrorInvalidValue;
+    const uint64_t xdims[3] = {(uint64_t)dpad, (uint64_t)rows, (uint64_t)k};
+    const uint32_t box_a[3] = {64, 128, 1}, box_b[3] = {64, 64, 1};
+    const uint64_t wdims[2] = {(uint64_t)dpad, (uint64_t)hidden};
+    const uint32_t wbox[2] = {64, 256}, wbox_h[2] = {64, 128};
+    const uint64_t hdims[3] = {(uint64_t)hpad, (uint64_t)rows, (uint64_t)k};
+    const uint64_t d1dims[3] = {(uint64_t)hidden, (uint64_t)rows, (uint64_t)k};
+    const uint64_t d2dims[3] = {64, (uint64_t)rows, (uint64_t)k};
+    // h in 128-row boxes (head: tmHa) and in 64-row boxes (backward operand: tmH); the same 128 x 64 box serves the
+    // head's loads of h and its stores of delta1 (tmD1s)
+    if (!make_map(&c.tmXa, Xb, 3, xdims, box_a) || !make_map(&c.tmXb, Xb, 3, xdims, box_b) ||
+        !make_map(&c.tmW, W1t, 2, wdims, wbox) || !make_map(&c.tmWh, W1t, 2, wdims, wbox_h) ||
+        !make_map(&c.tmH, H, 3, hdims, box_b) || !make_map(&c.tmHa, H, 3, hdims, box_a) ||
+        !make_map(&c.tmD1, D1, 3, d1dims, box_b) || !make_map(&c.tmD1s, D1, 3, d1dims, box_a) ||
+        !make_map(&c.tmD2, D2, 3, d2dims, box_b))
+      return cudaErrorInvalidValue;
+    if (head_tc) {
+      const uint64_t w2tdims[2] = {(uint64_t)hidden, 16}, w2kdims[2] = {64, (uint64_t)hidden};
+      const uint32_t box_w2t[2] = {64, 16}, box_w2k[2] = {64, 256};
+      if (!make_map(&c.tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&c.tmW2k, W2k, 2, w2kdims, box_w2k))
+        return cudaErrorInvalidValue;
+    }
+    c.k = k; c.rows = rows; c.d = d; c.hidden = hidden; c.C = C; c.sms = sms; c.Xb = Xb; c.scratch = scratch;
+    c.valid = true;
+  }
+  const int max_slots = c.max_slots;
+  float *slots = reinterpret_cast<float *>(ptr); ptr += up256((size_t)k * max_slots * ((size_t)hidden * C + C) * 4);
+  float *G = reinterpret_cast<float *>(ptr);
+  *G_out = G;
+  *G_ld = (long long)lpad;
+  const float *W1 = theta, *b1 = theta + (size_t)d * hidden, *W2 = b1 + hidden, *b2 = W2 + (size_t)hidden * C;
+
   MlpPrepParams pp;
-  pp.X = X; pp.Xb = Xb; pp.rows_total = (long long)kr; pp.d = d; pp.dpad = dpad;
+  pp.X = X; pp.Xb = Xb; pp.rows_total = prepared ? 0 : (long long)kr; pp.d = d; pp.dpad = dpad;
   pp.W1 = W1; pp.b1 = b1; pp.W1t = W1t; pp.hidden = hidden;
   pp.W2 = W2; pp.C = C; pp.W2t = W2t; pp.W2k = W2k;
   pp.tr_bx = (hidden + 31) / 32; pp.tr_blocks = pp.tr_bx * ((dpad + 31) / 32);
   pp.w2_blocks = head_tc ? (hidden * 64 + 255) / 256 : 0;
-  const long long groups = (long long)kr * (dpad / 8);
+  const long long groups = pp.rows_total * (dpad / 8);
   launch_k(mlp_prep_kernel, (unsigned)(pp.tr_blocks + pp.w2_blocks + (groups + 255) / 256), 256, 0, stream, pp);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-
-  e = cudaFuncSetAttribute(fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFwd);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc);
   if (e != cudaSuccess) return e;
 
   // H = relu([X 1] [W1; b1]), with its own column of ones behind the hidden units
@@ -1709,34 +1824,24 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   p.y = y; p.out = H; p.out_ld = hpad; p.ones_col = fuse_w2 ? -1 : hidden; p.status = status;
   const bool pair = (hidden % 256 == 0) && sms >= 2;  // CTA pairs: 256 rows per tile, half of W1^T per CTA
   if (pair) {
-    CUtensorMap tmWh;
-    const uint32_t wbox_h[2] = {64, 128};
-    if (!make_map(&tmWh, W1t, 2, wdims, wbox_h)) return cudaErrorInvalidValue;
     p.row_blocks = (rows + 255) / 256;
     p.num_tiles = k * p.row_blocks * p.n_tiles;
-    e = launch_pair(fwd_pair_kernel<1>, kFwdThreads, p.num_tiles, sms, tmXa, tmWh, p, stream);
+    e = launch_pair(fwd_pair_kernel<1>, kFwdThreads, p.num_tiles, sms, c.tmXa, c.tmWh, p, stream);
   } else {
-    launch_k(fwd_kernel<1>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, tmXa, tmW, p);
+    if ((e = ensure_smem_attr(fwd_kernel<1>, kSmemFwd)) != cudaSuccess) return e;
+    launch_k(fwd_kernel<1>, p.num_tiles < sms ? p.num_tiles : sms, kFwdThreads, kSmemFwd, stream, c.tmXa, c.tmW, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
 
   HeadSlots head_slots = {};
   if (head_tc) {
-    CUtensorMap tmW2t, tmW2k, tmD1s;
-    const uint64_t w2tdims[2] = {(uint64_t)hidden, 16}, w2kdims[2] = {64, (uint64_t)hidden};
-    const uint32_t box_w2t[2] = {64, 16}, box_w2k[2] = {64, 256};
-    if (!make_map(&tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&tmW2k, W2k, 2, w2kdims, box_w2k) ||
-        !make_map(&tmD1s, D1, 3, d1dims, box_a))
-      return cudaErrorInvalidValue;
     HeadTcParams hp;
     hp.hidden = hidden; hp.C = C; hp.rows = rows; hp.tiles_per_part = tpp; hp.num_tiles = k * tpp;
     hp.b2 = b2; hp.y = y; hp.D2 = D2; hp.fuse = fuse_w2 ? 1 : 0;
     hp.slots = slots; hp.max_slots = max_slots; hp.status = status;
-    e = cudaFuncSetAttribute(mlp_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_tc_smem);
-    if (e != cudaSuccess) return e;
-    // the same 128 x 64 box serves the loads of h and the stores of delta1
-    launch_k(mlp_head_tc_kernel, hgrid, kHeadTcThreads, head_tc_smem, stream, tmHa, tmW2t, tmW2k, tmD1s, hp);
+    if ((e = ensure_smem_attr(mlp_head_tc_kernel, (int)head_tc_smem)) != cudaSuccess) return e;
+    launch_k(mlp_head_tc_kernel, hgrid, kHeadTcThreads, head_tc_smem, stream, c.tmHa, c.tmW2t, c.tmW2k, c.tmD1s, hp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (fuse_w2) {
       head_slots.slots = slots; head_slots.max_slots = max_slots; head_slots.wstride = hidden * C + C;
@@ -1753,7 +1858,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     const unsigned head_blocks = (unsigned)((kr + kHeadRows - 1) / kHeadRows);
 #define NGC_LAUNCH_HEAD(CP)                                                                                       \
   do {                                                                                                            \
-    e = cudaFuncSetAttribute(mlp_head_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem);   \
+    e = ensure_smem_attr(mlp_head_kernel<CP>, (int)head_smem);                                                    \
     if (e != cudaSuccess) return e;                                                                               \
     launch_k(mlp_head_kernel<CP>, head_blocks, kHeadThreads, head_smem, stream, H, hpad, hidden, C, W2, b2, y,          \
                                                                           (long long)kr, D1, D2);                 \
@@ -1780,18 +1885,20 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
     wp.num_units = k * wp.m_tiles * wp.n_passes; wp.num_k = (rows + 63) / 64;
     wp.n_total = d + 1; wp.out = G; wp.out_batch = lpad; wp.out_ld = hidden; wp.status = status;
     wp.side = head_slots;
-    e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, tmD1, tmXb, wp, stream, kSmemWide);
+    e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, c.tmD1, c.tmXb, wp, stream, kSmemWide);
   } else {
-    launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmXb, tmD1, t);
+    if ((e = ensure_smem_attr(tn_gemm_kernel, kSmemTc)) != cudaSuccess) return e;
+    launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, c.tmXb, c.tmD1, t);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess || fuse_w2) return e;
   // [dW2; db2] = [h 1]^T delta2
+  if ((e = ensure_smem_attr(tn_gemm_kernel, kSmemTc)) != cudaSuccess) return e;
   t.m_tiles = (hidden + 1 + 127) / 128; t.n_tiles = 1; t.num_tiles = k * t.m_tiles;
   t.N = 16; t.nbox = 1;
   t.m_store = hidden + 1; t.n_store = C;
   t.out = G + (size_t)d * hidden + hidden; t.out_batch = lpad; t.out_ld = C;
-  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, tmH, tmD2, t);
+  launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, c.tmH, c.tmD2, t);
   return cudaGetLastError();
 }
 

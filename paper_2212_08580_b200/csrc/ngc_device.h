@@ -66,18 +66,28 @@ cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long
                                int s, long long d, void *coded, int coded_dtype, cudaStream_t stream,
                                const EncodeDecodeArgs *dec = nullptr);
 
+// Per-plan state of the dense launchers (created on first use): tensor maps and derived sizes of the last
+// problem, so that a repeated call encodes nothing on the host, and the data prepared once for the MLP.
+struct DenseState;
+void dense_state_free(DenseState *st);
+size_t dense_state_bytes(const DenseState *st);  // device memory it owns
+
 // MLP (one hidden ReLU layer, softmax cross-entropy) partial gradients on the tensor cores (X fp32):
 // G[k][*G_ld] fp32 inside `scratch`, each row holding [dW1, db1, dW2, db2].
 size_t mlp_scratch_bytes(int k, int rows, int d, int hidden, int C);
 int mlp_launch_count(int hidden);  // kernels one gradient + encode call launches
 cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const float *X, const int *y, const float *theta,
                             unsigned char *scratch, float **G_out, long long *G_ld, int *status, int sms,
-                            cudaStream_t stream);
+                            cudaStream_t stream, DenseState **state);
+// bf16 copy [X 1] of the MLP's data matrix, made once and used by every later launch_mlp_grad on the same X
+// (Section II-C: the data is assigned before training starts); X == nullptr drops it.
+cudaError_t prepare_mlp_data(DenseState **state, int k, int rows, int d, const float *X, cudaStream_t stream);
 
 // Softmax-regression partial gradients on the tensor cores (X bf16): G[k][d*C] fp32 inside `scratch`.
 size_t softmax_scratch_bytes(int k, int rows, int d, int C);
 cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, const int *y, const float *W,
-                                unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream);
+                                unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream,
+                                DenseState **state);
 
 // Monte Carlo of the stopping rule (Section IV): latency (gamma + eps + decode instant, +inf if never) and
 // chosen level (-1 if none) of `trials` seeded straggler patterns, into device buffers.

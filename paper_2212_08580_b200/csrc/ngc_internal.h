@@ -36,6 +36,7 @@ struct ngc_plan_s {
   int a_batch_cap = 0;
   int *d_status = nullptr;     // [0] timeout flag, [1] scratch
   double *d_maxres = nullptr;  // largest residual seen by asynchronous decodes
+  void *dense_state = nullptr; // ngc::DenseState*: cached tensor maps of the dense launchers, data prepared once
   void *d_gpart = nullptr;     // per-chunk partial decodes of the fused encode + decode (dense models)
   size_t gpart_bytes = 0;
   // ngc_step solves the decoding vector on a stream of its own while the gradients are computed

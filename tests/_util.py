@@ -41,3 +41,35 @@ def rel_l2(a, b):
 
 def coded_torch_dtype(code: int):
     return torch.float64 if code == ngc.NGC_F64 else torch.float32
+
+
+def block_rel_l2(got, want, ncols, block_rows=128, block_cols=256):
+    """Largest relative L2 error over the block_rows x block_cols blocks of the (len / ncols) x ncols view
+    of two vectors: a wrong strip at a ragged tile edge, or one misplaced output tile, cannot hide in the
+    norm of the whole gradient.  Blocks follow the kernels' output tiling (128 rows x 256 columns)."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1, ncols)
+    want = np.asarray(want, dtype=np.float64).reshape(-1, ncols)
+    worst = 0.0
+    for r0 in range(0, got.shape[0], block_rows):
+        for c0 in range(0, ncols, block_cols):
+            g, w = got[r0:r0 + block_rows, c0:c0 + block_cols], want[r0:r0 + block_rows, c0:c0 + block_cols]
+            worst = max(worst, float(np.linalg.norm(g - w) / max(np.linalg.norm(w), 1e-300)))
+    return worst
+
+
+def max_abs_scaled(got, want):
+    """Largest absolute error relative to the largest magnitude of the expected values."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    return float(np.max(np.abs(got - want)) / max(np.max(np.abs(want)), 1e-300))
+
+
+def assert_dense_close(got, want, ncols, tol, what=""):
+    """Whole-vector relative L2, every 128 x 256 block of the matrix view, and the largest single error."""
+    assert np.isfinite(np.asarray(got)).all(), what
+    e = rel_l2(got, want)
+    assert e < tol, (what, "rel L2", e)
+    b = block_rel_l2(got, want, ncols)
+    assert b < tol, (what, "worst 128 x 256 block", b)
+    m = max_abs_scaled(got, want)
+    assert m < tol, (what, "max abs / max |want|", m)

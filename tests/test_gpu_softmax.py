@@ -6,7 +6,7 @@ import torch
 import ngc_inputs
 import paper_2212_08580_b200 as ngc
 from oracle import ngc_oracle as orc
-from tests._util import coded_torch_dtype, group_G, model_of, oracle_G, rel_l2
+from tests._util import assert_dense_close, coded_torch_dtype, group_G, model_of, oracle_G, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -53,10 +53,11 @@ def test_softmax_grad_encode_decode_match_oracle(n, levels, rows, d, C, q):
         want = orc.encode(pl["B"][layer], G)
         got = coded.cpu().numpy()
         for i in range(n):
-            assert rel_l2(got[i], want[i]) < TOL, (layer, i, rel_l2(got[i], want[i]))
+            # the whole row, every 128-feature x 256-class block of it, and the largest single error
+            assert_dense_close(got[i], want[i], C, TOL, (layer, i))
         for trial in range(2):
             stragglers = rng.choice(n, size=s, replace=False) if trial else np.arange(s)
             S = np.array(sorted(set(range(n)) - set(int(v) for v in stragglers)), dtype=np.int32)
             p.decode(layer, S, coded, cdt, l, grad)
             torch.cuda.synchronize()
-            assert rel_l2(grad.cpu().numpy(), g_full) < TOL
+            assert_dense_close(grad.cpu().numpy(), g_full, C, TOL, (layer, "decoded"))
