@@ -11,7 +11,9 @@
 // Warp roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (+ tensor-memory owner), warps 2-5
 // epilogue (one accumulator row per thread).  Two 256-column accumulators let the epilogue of one
 // tile overlap the contraction of the next.
+#include <mutex>
 #include <new>
+#include <vector>
 
 #include "ngc_device.h"
 #include "ngc_pdl.cuh"
@@ -1466,16 +1468,29 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   pair_teardown(warp, tmem_base, failed, p.status);
 }
 
-// The opt-in shared-memory size of a kernel is set once per device, not on every launch.
+// The opt-in shared-memory size of a kernel is set once per device and kernel, not on every launch.
+struct SmemAttrDone {
+  const void *kern;
+  int dev, bytes;
+};
 template <typename Kern>
 cudaError_t ensure_smem_attr(Kern kern, int smem_bytes) {
-  static int done_bytes[64] = {};  // per device: the size already set for this kernel (one static per instantiation)
+  static std::mutex mu;
+  static std::vector<SmemAttrDone> done;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (dev >= 0 && dev < 64 && done_bytes[dev] >= smem_bytes) return cudaSuccess;
+  const void *key = reinterpret_cast<const void *>(kern);  // kernels of one signature share this template instance
+  std::lock_guard<std::mutex> lock(mu);
+  for (auto &d : done)
+    if (d.kern == key && d.dev == dev) {
+      if (d.bytes >= smem_bytes) return cudaSuccess;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+      if (e == cudaSuccess) d.bytes = smem_bytes;
+      return e;
+    }
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-  if (e == cudaSuccess && dev >= 0 && dev < 64) done_bytes[dev] = smem_bytes;
+  if (e == cudaSuccess) done.push_back({key, dev, smem_bytes});
   return e;
 }
 

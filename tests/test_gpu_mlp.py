@@ -54,6 +54,7 @@ def test_mlp_grad_encode_decode_match_oracle(n, levels, rows, d, hidden, C, q):
         mask = (X[j].cpu().bfloat16().double() @ W1 + b1 > 0).numpy()
         Gm.append(orc.grad_mlp(X[j].double().cpu().numpy(), y[j].cpu().numpy(), th.numpy(), hidden, C, relu_mask=mask))
     Gm = group_G(np.stack(Gm), q)
+    gm_full = Gm.sum(axis=0)
     l = w.n_params
     cdt = p.coded_dtype(m)
     coded = torch.empty((n, l), dtype=coded_torch_dtype(cdt), device="cuda")
@@ -89,7 +90,12 @@ def test_mlp_grad_encode_decode_match_oracle(n, levels, rows, d, hidden, C, q):
             torch.cuda.synchronize()
             gd = grad.cpu().numpy()
             assert rel_l2(gd, g_full) < TOL
-            assert_dense_close(gd[:o1], g_full[:o1], hidden, TOL, (layer, "decoded dW1"))
+            # the whole decoded gradient against the pure fp64 oracle at TOL (above); its first-layer part alone
+            # carries the ReLU decisions that flip under bf16 operands (a flipped unit of one sample is an O(1)
+            # error in single entries of dW1, which weighs most when partitions have few rows): bounded like the
+            # coded rows, and checked tile by tile and entry by entry with the decision matched
+            assert rel_l2(gd[:o2], g_full[:o2]) < TOL_PURE_ROW
+            assert_dense_close(gd[:o1], gm_full[:o1], hidden, TOL, (layer, "decoded dW1, decision matched"))
             assert_dense_close(gd[o2:o3], g_full[o2:o3], C, TOL, (layer, "decoded dW2"))
 
 
