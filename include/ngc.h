@@ -199,6 +199,31 @@ int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta
                   const void *y_host, const double *task_times_host, float *grad_host, ngc_step_info_t *info);
 
 /*
+ * One problem sharded over several GPUs (Section II-C: the data is split into row blocks that independent
+ * workers hold; here a GPU holds a contiguous block of partition groups and simulates the workers that start
+ * in it).  A rank calls, per iteration:
+ *   1. ngc_shard_gradients on its own partitions: G_dev[j] = g_j for its n_local groups (fp32, row stride ld
+ *      >= l, a multiple of 4; X_local_dev / y_local_dev point at the rank's first partition and hold
+ *      n_local * q partitions);
+ *   2. (caller) fetches the partial gradients of the next s_l groups in cyclic order from the ranks that
+ *      own them and appends them: G_window_dev = [own n_local rows; s_l halo rows];
+ *   3. ngc_shard_encode_decode: the coded gradients x_i of workers first_worker .. first_worker + n_local - 1
+ *      (coded_dev rows 0 .. n_local - 1; it needs room for n_local + s_l rows, the rest is scratch), and this
+ *      rank's share of the decode, sum over its responsive workers of a_i x_i with a the decoding vector of
+ *      the WHOLE responsive set S_host (every rank passes the same S).  partial_dev receives l values in the
+ *      coded dtype, unrounded when that is fp64: the code is ill-conditioned, the shares are large and
+ *      cancel, so they are added across ranks before anything is rounded to fp32;
+ *   4. (caller) one all-reduce (sum) of partial_dev over the ranks gives the decoded gradient.
+ * Results equal those of ngc_grad_encode + ngc_decode on one GPU up to summation order.  n_local + s_l <=
+ * NGC_MAX_N.  Asynchronous on the stream except for a short synchronisation in step 3.
+ */
+int ngc_shard_gradients(ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev, const void *X_local_dev,
+                        const void *y_local_dev, int n_local, float *G_dev, int64_t ld, void *cuda_stream);
+int ngc_shard_encode_decode(ngc_plan_t *plan, const ngc_model_t *model, int layer, int first_worker, int n_local,
+                            const float *G_window_dev, int64_t ld, const int32_t *S_host, int nS, void *coded_dev,
+                            void *partial_dev, void *cuda_stream);
+
+/*
  * Gradient-descent update of Eq. 1: theta <- theta - step * g with step = eta_t / m (the 1/m of Eq. 1 is
  * the caller's: the decoded gradient is a plain sum).  theta_dev and grad_dev hold l floats; asynchronous
  * on the stream, so it can be enqueued right behind ngc_step.

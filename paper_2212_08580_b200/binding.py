@@ -69,6 +69,8 @@ def load_library() -> C.CDLL:
         "ngc_coded_dtype": (i32, [vp, P(Model)]),
         "ngc_select": (i32, [vp, P(dbl), P(StepInfo)]),
         "ngc_prepare_data": (i32, [vp, P(Model), vp, vp]),
+        "ngc_shard_gradients": (i32, [vp, P(Model), vp, vp, vp, i32, vp, i64, vp]),
+        "ngc_shard_encode_decode": (i32, [vp, P(Model), i32, i32, i32, vp, i64, P(C.c_int32), i32, vp, vp, vp]),
         "ngc_grad_encode": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp]),
         "ngc_grad_encode_static": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp, vp]),
         "ngc_decode_vector": (i32, [vp, i32, P(C.c_int32), i32, P(dbl)]),
@@ -215,6 +217,17 @@ class Plan:
         """ngc_prepare_data: what the library derives from the data matrix alone, made once (X=None drops it)."""
         self._check(self._lib.ngc_prepare_data(self._h, C.byref(model), _addr(X) if X is not None else None, stream),
                     "ngc_prepare_data")
+
+    def shard_gradients(self, model: Model, theta, X_local, y_local, n_local: int, G, ld: int, stream: int = 0):
+        self._check(self._lib.ngc_shard_gradients(self._h, C.byref(model), _addr(theta), _addr(X_local), _addr(y_local),
+                                                  n_local, _addr(G), ld, stream), "ngc_shard_gradients")
+
+    def shard_encode_decode(self, model: Model, layer: int, first_worker: int, n_local: int, G_window, ld: int, S,
+                            coded, partial, stream: int = 0):
+        S = np.ascontiguousarray(S, dtype=np.int32)
+        self._check(self._lib.ngc_shard_encode_decode(self._h, C.byref(model), layer, first_worker, n_local,
+                                                      _addr(G_window), ld, _iptr(S), len(S), _addr(coded),
+                                                      _addr(partial), stream), "ngc_shard_encode_decode")
 
     def grad_encode(self, model: Model, theta, X, y, layer: int, coded, stream: int = 0):
         self._check(self._lib.ngc_grad_encode(self._h, C.byref(model), _addr(theta), _addr(X), _addr(y), layer,

@@ -149,6 +149,8 @@ void ngc_plan_destroy(ngc_plan_t *p) {
     cudaFree(p->d_status);
     cudaFree(p->d_maxres);
     cudaFree(p->d_gpart);
+    cudaFree(p->d_shard_coef);
+    cudaFree(p->d_shard_a);
     cudaFree(p->st_X);
     cudaFree(p->st_y);
     cudaFree(p->st_theta);
@@ -209,6 +211,80 @@ int encode_dense(ngc_plan_t *p, const ngc::RowSplit &split, const float *G, long
   return NGC_OK;
 }
 
+// Where the gradient kernels left the partial gradients of the partition groups: fp32 [group][slot][ld], the
+// slots of a group to be added up in order (see RowSplit).
+struct PartialGrads {
+  ngc::RowSplit split;
+  const float *ws;
+  long long ld;
+  int launches;
+};
+
+// Partial gradients g_j of `n_groups` consecutive partition groups (q partitions each) whose data start at X / y:
+// the gradient kernels of the model kind, into the plan's scratch.  The whole problem is n_groups = n; a shard of
+// it passes fewer.
+int partial_gradients(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int n_groups,
+                      cudaStream_t stream, PartialGrads *out) {
+  int rc;
+  const int sms = ngc::device_sm_count();
+  if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
+  const int k = n_groups * p->q;
+  if (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) {
+    const int vec = (m->x_dtype == NGC_F32) ? 4 : 8;
+    if (m->d % vec != 0 || m->d / vec > 4 * 512) return NGC_ERR_INVALID;  // rows must be whole 16-byte vectors
+    out->split = ngc::make_row_split(n_groups, (long long)p->q * m->rows_per_partition, sms);
+    rc = ensure_ws(p, (size_t)n_groups * out->split.P * m->d * sizeof(float));
+    if (rc != NGC_OK) return rc;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_gemv_pair(*m, out->split, X, static_cast<const float *>(y), static_cast<const float *>(theta),
+                                      static_cast<float *>(p->ws), p->d_status, stream));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    out->ws = static_cast<const float *>(p->ws);
+    out->ld = m->d;
+    out->launches = 1;
+    return NGC_OK;
+  }
+  // dense models: one scratch slot per partition, a group is q consecutive partitions
+  out->split.T = k; out->split.rows_g = p->q; out->split.grid = k; out->split.P = p->q;
+  float *G = nullptr;
+  if (m->kind == NGC_SOFTMAX) {
+    if (m->x_dtype != NGC_BF16 || m->n_classes % 16 != 0 || m->n_classes < 16 || m->n_classes > 256 || m->d % 8 != 0)
+      return NGC_ERR_INVALID;
+    rc = ensure_ws(p, ngc::softmax_scratch_bytes(k, m->rows_per_partition, m->d, m->n_classes));
+    if (rc != NGC_OK) return rc;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_softmax_grad(k, m->rows_per_partition, m->d, m->n_classes, X, static_cast<const int *>(y),
+                                         static_cast<const float *>(theta), static_cast<unsigned char *>(p->ws), &G,
+                                         p->d_status, sms, stream,
+                                         reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    out->ws = G;
+    out->ld = ngc_num_params(m);
+    out->launches = 3;
+    return NGC_OK;
+  }
+  if (m->kind == NGC_MLP) {
+    if (m->x_dtype != NGC_F32) return NGC_ERR_INVALID;
+    const int h = m->hidden, C = m->n_classes;
+    if (m->d % 8 != 0 || h % 16 != 0 || h < 16 || h > 512 || (h > 256 && h % 256 != 0) || C < 1 || C > 16)
+      return NGC_ERR_INVALID;
+    rc = ensure_ws(p, ngc::mlp_scratch_bytes(k, m->rows_per_partition, m->d, h, C));
+    if (rc != NGC_OK) return rc;
+    long long ldG = 0;
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    NGC_CUDA(p, ngc::launch_mlp_grad(k, m->rows_per_partition, m->d, h, C, static_cast<const float *>(X),
+                                     static_cast<const int *>(y), static_cast<const float *>(theta),
+                                     static_cast<unsigned char *>(p->ws), &G, &ldG, p->d_status, sms, stream,
+                                     reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
+    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
+    out->ws = G;
+    out->ld = ldG;
+    out->launches = ngc::mlp_launch_count(h) - 1;
+    return NGC_OK;
+  }
+  return NGC_ERR_INVALID;
+}
+
 int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
                      void *coded, void *cuda_stream, DecodeHook *hook) {
   if (hook) hook->fused = false;
@@ -221,75 +297,90 @@ int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, con
   if (rc != NGC_OK) return rc;
   const int cdt = ngc_coded_dtype(p, m);
   const ngc_level_t &lv = p->lv[layer];
-
+  PartialGrads pg;
+  if ((rc = partial_gradients(p, m, theta, X, y, p->n, stream, &pg)) != NGC_OK) return rc;
   if (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) {
-    const int vec = (m->x_dtype == NGC_F32) ? 4 : 8;
-    if (m->d % vec != 0 || m->d / vec > 4 * 512) return NGC_ERR_INVALID;  // rows must be whole 16-byte vectors
-    const int sms = ngc::device_sm_count();
-    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
-    const ngc::RowSplit split = ngc::make_row_split(p->n, (long long)p->q * m->rows_per_partition, sms);
-    rc = ensure_ws(p, (size_t)p->n * split.P * m->d * sizeof(float));
-    if (rc != NGC_OK) return rc;
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    NGC_CUDA(p, ngc::launch_gemv_pair(*m, split, X, static_cast<const float *>(y), static_cast<const float *>(theta),
-                                      static_cast<float *>(p->ws), p->d_status, stream));
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    NGC_CUDA(p, ngc::launch_combine_encode(split, static_cast<const float *>(p->ws), lv.d_coef, p->n, lv.s, m->d,
-                                           coded, cdt, stream));
-    p->launches += 2;
-    return NGC_OK;
+    NGC_CUDA(p, ngc::launch_combine_encode(pg.split, pg.ws, lv.d_coef, p->n, lv.s, m->d, coded, cdt, stream));
+  } else {
+    if ((rc = encode_dense(p, pg.split, pg.ws, pg.ld, lv, ngc_num_params(m), coded, cdt, stream, hook)) != NGC_OK)
+      return rc;
   }
-  if (m->kind == NGC_SOFTMAX) {
-    if (m->x_dtype != NGC_BF16 || m->n_classes % 16 != 0 || m->n_classes < 16 || m->n_classes > 256 || m->d % 8 != 0)
-      return NGC_ERR_INVALID;
-    const int sms = ngc::device_sm_count();
-    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
-    rc = ensure_ws(p, ngc::softmax_scratch_bytes(p->k, m->rows_per_partition, m->d, m->n_classes));
-    if (rc != NGC_OK) return rc;
-    float *G = nullptr;
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    NGC_CUDA(p, ngc::launch_softmax_grad(p->k, m->rows_per_partition, m->d, m->n_classes, X, static_cast<const int *>(y),
-                                         static_cast<const float *>(theta), static_cast<unsigned char *>(p->ws), &G,
-                                         p->d_status, sms, stream,
-                                         reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    // G is [n][q][l]: group g of q consecutive partitions, one scratch slot per partition
-    ngc::RowSplit split;
-    split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
-    const long long l = ngc_num_params(m);
-    if ((rc = encode_dense(p, split, G, l, lv, l, coded, cdt, stream, hook)) != NGC_OK) return rc;
-    p->launches += 4;
-    return NGC_OK;
-  }
-  if (m->kind == NGC_MLP) {
-    if (m->x_dtype != NGC_F32) return NGC_ERR_INVALID;
-    const int h = m->hidden, C = m->n_classes;
-    if (m->d % 8 != 0 || h % 16 != 0 || h < 16 || h > 512 || (h > 256 && h % 256 != 0) || C < 1 || C > 16)
-      return NGC_ERR_INVALID;
-    const int sms = ngc::device_sm_count();
-    if (sms <= 0) { p->last_cuda = (int)cudaErrorNoDevice; return NGC_ERR_CUDA; }
-    rc = ensure_ws(p, ngc::mlp_scratch_bytes(p->k, m->rows_per_partition, m->d, h, C));
-    if (rc != NGC_OK) return rc;
-    float *G = nullptr;
-    long long ldG = 0;
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    NGC_CUDA(p, ngc::launch_mlp_grad(p->k, m->rows_per_partition, m->d, h, C, static_cast<const float *>(X),
-                                     static_cast<const int *>(y), static_cast<const float *>(theta),
-                                     static_cast<unsigned char *>(p->ws), &G, &ldG, p->d_status, sms, stream,
-                                     reinterpret_cast<ngc::DenseState **>(&p->dense_state)));
-    if ((rc = profile_mark(p, stream)) != NGC_OK) return rc;
-    ngc::RowSplit split;
-    split.T = p->k; split.rows_g = p->q; split.grid = p->k; split.P = p->q;
-    if ((rc = encode_dense(p, split, G, ldG, lv, ngc_num_params(m), coded, cdt, stream, hook)) != NGC_OK) return rc;
-    p->launches += ngc::mlp_launch_count(h);
-    return NGC_OK;
-  }
-  return NGC_ERR_INVALID;
+  p->launches += pg.launches + 1;
+  return NGC_OK;
 }
 
 }  // namespace
 
 extern "C" {
+
+// ---- one problem sharded over several GPUs (Section II-C: the workers, each with its partitions, are independent)
+
+int ngc_shard_gradients(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X_local, const void *y_local,
+                        int n_local, float *G, int64_t ld, void *cuda_stream) {
+  if (!p || !theta || !X_local || !y_local || !G || n_local < 1 || n_local > p->n) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  const int64_t l = ngc_num_params(m);
+  if (ld < l || ld % 4 != 0 || !aligned16(X_local) || !aligned16(theta) || !aligned16(G)) return NGC_ERR_INVALID;
+  if ((rc = ensure_tables(p)) != NGC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  PartialGrads pg;
+  if ((rc = partial_gradients(p, m, theta, X_local, y_local, n_local, stream, &pg)) != NGC_OK) return rc;
+  NGC_CUDA(p, ngc::launch_sum_slots(pg.split, n_local, pg.ws, pg.ld, l, G, ld, stream));
+  p->launches += pg.launches + 1;
+  return NGC_OK;
+}
+
+int ngc_shard_encode_decode(ngc_plan_t *p, const ngc_model_t *m, int layer, int first_worker, int n_local,
+                            const float *G_window, int64_t ld, const int32_t *S, int nS, void *coded, void *partial,
+                            void *cuda_stream) {
+  if (!p || !G_window || !coded || !partial || layer < 0 || layer >= p->L) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  const ngc_level_t &lv = p->lv[layer];
+  const int n = p->n, s = lv.s, rows = n_local + s;  // the shard's workers, then s rows that only pad the windows
+  if (first_worker < 0 || first_worker >= n || n_local < 1 || n_local > n || rows > NGC_MAX_N) return NGC_ERR_INVALID;
+  const int64_t l = ngc_num_params(m);
+  if (ld < l || ld % 4 != 0 || !aligned16(G_window) || !aligned16(coded) || !aligned16(partial)) return NGC_ERR_INVALID;
+  ngc::MaskArg mask;
+  if ((rc = pack_set(p, layer, S, nS, mask.w)) != NGC_OK) return rc;
+  if ((rc = ensure_tables(p)) != NGC_OK) return rc;
+  if ((rc = ensure_batch(p, 1)) != NGC_OK) return rc;
+  if (!p->d_shard_coef) {
+    NGC_CUDA(p, cudaMalloc(&p->d_shard_coef, (size_t)NGC_MAX_N * (NGC_MAX_S + 1) * sizeof(double)));
+    NGC_CUDA(p, cudaMalloc(&p->d_shard_a, (size_t)NGC_MAX_N * sizeof(double)));
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // Rows first_worker .. first_worker + n_local - 1 of B (window form), then s all-zero rows: the encode kernels
+  // index the partial gradients cyclically over `rows` entries, and only the zero rows ever wrap.
+  p->shard_coef_host.assign((size_t)rows * (s + 1), 0.0);
+  for (int r = 0; r < n_local; ++r) {
+    const int i = (first_worker + r) % n;
+    for (int t = 0; t <= s; ++t) p->shard_coef_host[(size_t)r * (s + 1) + t] = lv.coef[(size_t)i * (s + 1) + t];
+  }
+  NGC_CUDA(p, cudaMemcpyAsync(p->d_shard_coef, p->shard_coef_host.data(), p->shard_coef_host.size() * sizeof(double),
+                              cudaMemcpyHostToDevice, stream));
+  NGC_CUDA(p, cudaStreamSynchronize(stream));  // the host vector is reused by the next call
+  const int cdt = ngc_coded_dtype(p, m);
+  ngc::RowSplit split;
+  split.T = rows; split.rows_g = 1; split.grid = rows; split.P = 1;
+  NGC_CUDA(p, ngc::launch_encode_long(split, G_window, ld, p->d_shard_coef, rows, s, l, coded, cdt, stream));
+  // the decoding vector of the whole responsive set; this shard applies the weights of its own workers
+  NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
+  NGC_CUDA(p, cudaMemsetAsync(p->d_shard_a, 0, (size_t)NGC_MAX_N * sizeof(double), stream));
+  const int head = (first_worker + n_local <= n) ? n_local : n - first_worker;  // workers before the index wraps
+  NGC_CUDA(p, cudaMemcpyAsync(p->d_shard_a, p->d_a + first_worker, (size_t)head * sizeof(double),
+                              cudaMemcpyDeviceToDevice, stream));
+  if (head < n_local)
+    NGC_CUDA(p, cudaMemcpyAsync(p->d_shard_a + head, p->d_a, (size_t)(n_local - head) * sizeof(double),
+                                cudaMemcpyDeviceToDevice, stream));
+  if (cdt == NGC_F64)
+    NGC_CUDA(p, ngc::launch_decode(coded, cdt, p->d_shard_a, rows, l, nullptr, stream, static_cast<double *>(partial)));
+  else
+    NGC_CUDA(p, ngc::launch_decode(coded, cdt, p->d_shard_a, rows, l, static_cast<float *>(partial), stream));
+  p->launches += 3;
+  return NGC_OK;
+}
 
 int ngc_prepare_data(ngc_plan_t *p, const ngc_model_t *m, const void *X, void *cuda_stream) {
   if (!p) return NGC_ERR_INVALID;

@@ -134,7 +134,8 @@ constexpr int kDecWarps = 8;
 
 template <typename CT, int V>
 __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
-                                                              int n, long long l, float *__restrict__ grad) {
+                                                              int n, long long l, float *__restrict__ grad,
+                                                              double *__restrict__ grad64) {
   pdl_sync();
   __shared__ double as[NGC_MAX_N];
   __shared__ double part[kDecWarps][32 * V];
@@ -168,7 +169,8 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__rest
       double sum = 0.0;
 #pragma unroll
       for (int w = 0; w < kDecWarps; ++w) sum += part[w][c];
-      grad[gc] = (float)sum;
+      if (grad64) grad64[gc] = sum;  // partial decode of one shard: added to the other shards' before rounding
+      else grad[gc] = (float)sum;
     }
   }
 }
@@ -178,7 +180,8 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_kernel(const CT *__rest
 // index order (a compacted list in shared memory), several loads in flight, no exchange between threads.
 template <typename CT, int V>
 __global__ void __launch_bounds__(256) decode_flat_kernel(const CT *__restrict__ coded, const double *__restrict__ a,
-                                                          int n, long long l, float *__restrict__ grad) {
+                                                          int n, long long l, float *__restrict__ grad,
+                                                          double *__restrict__ grad64) {
   pdl_sync();
   __shared__ double as[NGC_MAX_N];
   __shared__ double wt[NGC_MAX_N];
@@ -210,6 +213,11 @@ __global__ void __launch_bounds__(256) decode_flat_kernel(const CT *__restrict__
 #pragma unroll
     for (int e = 0; e < V; ++e) acc[e] = fma(w, (double)v[e], acc[e]);
   }
+  if (grad64) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) grad64[col + e] = acc[e];
+    return;
+  }
   float *dst = grad + col;
   if (V == 4 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
     *reinterpret_cast<float4 *>(dst) = make_float4((float)acc[0], (float)acc[V > 1 ? 1 : 0], (float)acc[V > 2 ? 2 : 0], (float)acc[V > 3 ? 3 : 0]);
@@ -224,16 +232,18 @@ __global__ void __launch_bounds__(256) decode_flat_kernel(const CT *__restrict__
 constexpr long long kDecodeFlatFrom = 1 << 16;  // parameters from which one thread per V columns fills the GPU
 
 template <typename CT, int V>
-cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, cudaStream_t stream) {
+cudaError_t run_decode(const void *coded, const double *a, int n, long long l, float *grad, double *grad64,
+                       cudaStream_t stream) {
   if (l >= kDecodeFlatFrom) {
     const long long per_block = 256 * V;
     launch_k(decode_flat_kernel<CT, V>, (unsigned)((l + per_block - 1) / per_block), 256, 0, stream, 
-        static_cast<const CT *>(coded), a, n, l, grad);
+        static_cast<const CT *>(coded), a, n, l, grad, grad64);
     return cudaGetLastError();
   }
   const long long per_block = 32 * V;
   const unsigned blocks = (unsigned)((l + per_block - 1) / per_block);
-  launch_k(decode_kernel<CT, V>, blocks, kDecWarps * 32, 0, stream, static_cast<const CT *>(coded), a, n, l, grad);
+  launch_k(decode_kernel<CT, V>, blocks, kDecWarps * 32, 0, stream, static_cast<const CT *>(coded), a, n, l, grad,
+           grad64);
   return cudaGetLastError();
 }
 
@@ -263,15 +273,15 @@ cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *
 }
 
 cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, double *grad64) {
   // widest vector that keeps every row 16- / 8-byte aligned
   if (coded_dtype == NGC_F64) {
-    if (l % 2 == 0) return run_decode<double, 2>(coded, a_dev, n, l, grad, stream);
-    return run_decode<double, 1>(coded, a_dev, n, l, grad, stream);
+    if (l % 2 == 0) return run_decode<double, 2>(coded, a_dev, n, l, grad, grad64, stream);
+    return run_decode<double, 1>(coded, a_dev, n, l, grad, grad64, stream);
   }
-  if (l % 4 == 0) return run_decode<float, 4>(coded, a_dev, n, l, grad, stream);
-  if (l % 2 == 0) return run_decode<float, 2>(coded, a_dev, n, l, grad, stream);
-  return run_decode<float, 1>(coded, a_dev, n, l, grad, stream);
+  if (l % 4 == 0) return run_decode<float, 4>(coded, a_dev, n, l, grad, grad64, stream);
+  if (l % 2 == 0) return run_decode<float, 2>(coded, a_dev, n, l, grad, grad64, stream);
+  return run_decode<float, 1>(coded, a_dev, n, l, grad, grad64, stream);
 }
 
 }  // namespace ngc

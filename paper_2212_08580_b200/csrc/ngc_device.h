@@ -42,9 +42,15 @@ struct MaskArg {
 cudaError_t launch_decode_solve(const ngc_plan_s &p, int layer, const uint64_t *masks_dev, MaskArg one, int batch,
                                 double *a_dev, double *resid_dev, double *maxres_dev, cudaStream_t stream);
 
-// g = sum_i a_i coded[i], a read from device memory (zeros skipped).
+// g = sum_i a_i coded[i], a read from device memory (zeros skipped).  With grad64 the sum is written there
+// unrounded instead of to grad (the partial decode of one shard of the workers).
 cudaError_t launch_decode(const void *coded, int coded_dtype, const double *a_dev, int n, long long l, float *grad,
-                          cudaStream_t stream);
+                          cudaStream_t stream, double *grad64 = nullptr);
+
+// G_out[g][c] = sum over the scratch slots of group g (fp64, slot order), c < l: the partial gradients themselves,
+// for a caller that exchanges them (sharded operation).  ws is [group][slot][ld_ws], G_out [group][ld_out].
+cudaError_t launch_sum_slots(const RowSplit &split, int n_groups, const float *ws, long long ld_ws, long long l,
+                             float *G_out, long long ld_out, cudaStream_t stream);
 
 // True when an SM that holds a CTA of the gradient kernel chosen for `m` can still take a one-warp block.
 bool gemv_pair_leaves_room(const ngc_model_t &m);

@@ -703,6 +703,30 @@ cudaError_t encode_long_typed(const RowSplit &split, const float *ws, long long 
 }
 }  // namespace
 
+namespace {
+__global__ void __launch_bounds__(256)
+sum_slots_kernel(const RowSplit split, const float *__restrict__ ws, long long ld_ws, long long l,
+                 float *__restrict__ G_out, long long ld_out) {
+  pdl_sync();
+  const long long col = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int g = blockIdx.y;
+  if (col >= l) return;
+  const int c0 = split_owner(split, (long long)g * split.rows_g);
+  const int c1 = split_owner(split, (long long)(g + 1) * split.rows_g - 1);
+  const float *src = ws + (size_t)g * split.P * ld_ws + col;
+  double acc = 0.0;
+  for (int pce = 0; pce <= c1 - c0; ++pce) acc += (double)__ldg(src + (size_t)pce * ld_ws);
+  G_out[(size_t)g * ld_out + col] = (float)acc;
+}
+}  // namespace
+
+cudaError_t launch_sum_slots(const RowSplit &split, int n_groups, const float *ws, long long ld_ws, long long l,
+                             float *G_out, long long ld_out, cudaStream_t stream) {
+  launch_k(sum_slots_kernel, dim3((unsigned)((l + 255) / 256), (unsigned)n_groups), 256, 0, stream, split, ws, ld_ws, l,
+           G_out, ld_out);
+  return cudaGetLastError();
+}
+
 // Encode for the dense models: ws holds [group][slot][ld_ws] fp32, every slot filled, ld_ws a multiple of 4 and >= d.
 cudaError_t launch_encode_long(const RowSplit &split, const float *ws, long long ld_ws, const double *d_coef, int n,
                                int s, long long d, void *coded, int coded_dtype, cudaStream_t stream,

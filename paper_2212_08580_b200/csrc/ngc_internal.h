@@ -36,6 +36,10 @@ struct ngc_plan_s {
   int a_batch_cap = 0;
   int *d_status = nullptr;     // [0] timeout flag, [1] scratch
   double *d_maxres = nullptr;  // largest residual seen by asynchronous decodes
+  // sharded operation: coefficient rows and decoding weights of the workers one shard holds
+  double *d_shard_coef = nullptr;  // NGC_MAX_N x (NGC_MAX_S + 1)
+  double *d_shard_a = nullptr;     // NGC_MAX_N
+  std::vector<double> shard_coef_host;
   void *dense_state = nullptr; // ngc::DenseState*: cached tensor maps of the dense launchers, data prepared once
   void *d_gpart = nullptr;     // per-chunk partial decodes of the fused encode + decode (dense models)
   size_t gpart_bytes = 0;
