@@ -777,11 +777,11 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       const bool valid = prow < p.rows;
       const long long row = (long long)j * p.rows + prow;
       if (part == 0) {
+        const int label = valid ? __ldg(p.y + row) : -1;  // on its way while the logits are being formed
         if (!mbar_wait(z_full, ph)) { failed = true; break; }
         tc_fence_after();
         float v[16];
         tmem_ld16(z_acc + lane_off, v);
-        const int label = valid ? p.y[row] : -1;
         float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
