@@ -161,6 +161,7 @@ void ngc_plan_destroy(ngc_plan_t *p) {
   for (void *e : p->ev) cudaEventDestroy(static_cast<cudaEvent_t>(e));
   if (p->ev_solved) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_solved));
   if (p->ev_decoded) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_decoded));
+  if (p->ev_grads) cudaEventDestroy(static_cast<cudaEvent_t>(p->ev_grads));
   if (p->side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(p->side_stream));
   delete p;
 }
@@ -176,6 +177,7 @@ struct DecodeHook {
   cudaEvent_t solved;
   float *grad;
   bool fused;
+  cudaEvent_t after_grads;  // if set: recorded on the caller's stream right behind the gradient kernels
 };
 
 int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y, int layer,
@@ -299,6 +301,7 @@ int grad_encode_impl(ngc_plan_t *p, const ngc_model_t *m, const void *theta, con
   const ngc_level_t &lv = p->lv[layer];
   PartialGrads pg;
   if ((rc = partial_gradients(p, m, theta, X, y, p->n, stream, &pg)) != NGC_OK) return rc;
+  if (hook && hook->after_grads) NGC_CUDA(p, cudaEventRecord(hook->after_grads, stream));
   if (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) {
     NGC_CUDA(p, ngc::launch_combine_encode(pg.split, pg.ws, lv.d_coef, p->n, lv.s, m->d, coded, cdt, stream));
   } else {
@@ -447,8 +450,9 @@ int ngc_decode(ngc_plan_t *p, int layer, const int32_t *S, int nS, const void *c
 // The decoding vector depends only on the responsive set, which is known before any gradient is:
 // ngc_step solves it on a stream of the plan's own, under the gradient kernels, and the decode on the
 // caller's stream waits for it.  The solve in turn waits for everything the caller's stream held when the
-// step was entered (the decode of the step before reads the same vector).  A capturing stream takes the
-// plain in-order path.
+// step was entered (the decode of the step before reads the same vector).  Where the gradient kernel leaves no
+// room on its SMs, the solve waits for that kernel instead and runs beside the small encode kernel.  A capturing
+// stream takes the plain in-order path.
 int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void *X, const void *y,
              const double *task_times, void *coded, float *grad, ngc_step_info_t *info, void *cuda_stream) {
   if (!p || !info) return NGC_ERR_INVALID;
@@ -465,7 +469,7 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
     p->overlap_kind = m->kind; p->overlap_d = m->d; p->overlap_dtype = m->x_dtype;
     p->overlap_ok = (m->kind == NGC_LSQ || m->kind == NGC_LOGISTIC) ? ngc::gemv_pair_leaves_room(*m) : true;
   }
-  if (!p->overlap_ok || cap != cudaStreamCaptureStatusNone || !coded || !grad || !aligned16(coded)) {
+  if (cap != cudaStreamCaptureStatusNone || !coded || !grad || !aligned16(coded)) {
     rc = ngc_grad_encode(p, m, theta, X, y, info->layer, coded, cuda_stream);
     if (rc != NGC_OK) return rc;
     return ngc_decode(p, info->layer, info->S, info->nS, coded, ngc_coded_dtype(p, m), ngc_num_params(m), grad,
@@ -478,26 +482,41 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
   if ((rc = ensure_batch(p, 1)) != NGC_OK) return rc;
   if (!p->side_stream) {
     cudaStream_t s2;
-    cudaEvent_t e1, e2;
+    cudaEvent_t e1, e2, e3;
     NGC_CUDA(p, cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking));
     p->side_stream = s2;
     NGC_CUDA(p, cudaEventCreateWithFlags(&e1, cudaEventDisableTiming));
     p->ev_solved = e1;
     NGC_CUDA(p, cudaEventCreateWithFlags(&e2, cudaEventDisableTiming));
     p->ev_decoded = e2;
+    NGC_CUDA(p, cudaEventCreateWithFlags(&e3, cudaEventDisableTiming));
+    p->ev_grads = e3;
   }
   cudaStream_t side = static_cast<cudaStream_t>(p->side_stream);
   cudaEvent_t solved = static_cast<cudaEvent_t>(p->ev_solved), decoded = static_cast<cudaEvent_t>(p->ev_decoded);
-  // Everything already queued on the caller's stream comes before the solve overwrites the vector: the decode
-  // of the step before, but also a replayed graph whose captured steps recorded no event.
-  NGC_CUDA(p, cudaEventRecord(decoded, stream));
-  NGC_CUDA(p, cudaStreamWaitEvent(side, decoded, 0));
-  NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
-  NGC_CUDA(p, cudaEventRecord(solved, side));
+  DecodeHook hook{solved, grad, false, nullptr};
+  if (p->overlap_ok) {
+    // Everything already queued on the caller's stream comes before the solve overwrites the vector: the decode
+    // of the step before, but also a replayed graph whose captured steps recorded no event.
+    NGC_CUDA(p, cudaEventRecord(decoded, stream));
+    NGC_CUDA(p, cudaStreamWaitEvent(side, decoded, 0));
+    NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
+    NGC_CUDA(p, cudaEventRecord(solved, side));
+  } else {
+    // The gradient kernel fills its SMs: the solve waits for it on the side stream and runs beside the small
+    // encode kernel instead of in line behind it.
+    hook.after_grads = static_cast<cudaEvent_t>(p->ev_grads);
+  }
   // Dense models: the encode kernel forms the decoded gradient from the coded rows as it writes them.
-  DecodeHook hook{solved, grad, false};
   rc = grad_encode_impl(p, m, theta, X, y, info->layer, coded, cuda_stream, &hook);
   if (rc != NGC_OK) return rc;
+  if (!p->overlap_ok) {
+    // (the gradient kernels of this step come after the decode of the step before on the caller's stream, so the
+    // vector is free by the time the event fires)
+    NGC_CUDA(p, cudaStreamWaitEvent(side, hook.after_grads, 0));
+    NGC_CUDA(p, ngc::launch_decode_solve(*p, info->layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, side));
+    NGC_CUDA(p, cudaEventRecord(solved, side));
+  }
   if (!hook.fused) {
     NGC_CUDA(p, cudaStreamWaitEvent(stream, solved, 0));
     NGC_CUDA(p, ngc::launch_decode(coded, ngc_coded_dtype(p, m), p->d_a, p->n, ngc_num_params(m), grad, stream));

@@ -47,6 +47,7 @@ struct ngc_plan_s {
   void *side_stream = nullptr; // cudaStream_t, non-blocking
   void *ev_solved = nullptr;   // cudaEvent_t: d_a holds the vector of the current step
   void *ev_decoded = nullptr;  // cudaEvent_t: the last decode has read d_a
+  void *ev_grads = nullptr;    // cudaEvent_t: the gradient kernels of the current step are done
   int overlap_kind = -1, overlap_d = -1, overlap_dtype = -1;  // model the answer below was taken for
   bool overlap_ok = false;     // the gradient kernel leaves room for the solve's warp on its SMs
   // staging for ngc_step_host
