@@ -324,13 +324,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     if (lane == 0) {
       int st = 0;
       uint32_t ph = 0;
+      const uint64_t stream_once = l2_evict_first_policy();  // the data matrix: read once by this kernel
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
         const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
           mbar_expect_tx(s.full[st], kStageBytes);
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
-          tma_load_3d(a, &tmX, kc * 64, rb * 128, j, s.full[st]);
+          tma_load_3d_hint(a, &tmX, kc * 64, rb * 128, j, s.full[st], stream_once);
           tma_load_2d(a + kABytes, &tmW, kc * 64, nt * 256, s.full[st]);
           if (++st == kFwdStages) { st = 0; ph ^= 1u; }
         }
@@ -680,11 +681,12 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
         for (int kc = 0; kc < nchunk; ++kc) tma_load_2d(smem_u32(w2t + kc * 2048), &tmW2t, kc * 64, 0, w_full);
         for (int hh = 0; hh < nhalf; ++hh) tma_load_2d(smem_u32(w2k + hh * 32768), &tmW2k, 0, hh * 256, w_full);
       }
+      const uint64_t stream_once = l2_evict_first_policy();  // h is read here for the last time
       auto load_group = [&](int tile, int g) {
         const int j = tile / tpp, rb = tile % tpp, c0 = g * 2, c1 = min(nchunk, c0 + 2);
         mbar_expect_tx(h_full[g], (uint32_t)(c1 - c0) * 16384u);
         for (int kc = c0; kc < c1; ++kc)
-          tma_load_3d(smem_u32(htile + kc * 16384), &tmH, kc * 64, rb * 128, j, h_full[g]);
+          tma_load_3d_hint(smem_u32(htile + kc * 16384), &tmH, kc * 64, rb * 128, j, h_full[g], stream_once);
       };
       for (int g = g0; g < ngroups; g += 2) load_group(t_begin, g);
       uint32_t ph = 0;
@@ -959,14 +961,15 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int st = 0;
       uint32_t ph = 0;
       const uint32_t tx = (uint32_t)(2 + p.nbox) * 8192u;
+      const uint64_t stream_once = l2_evict_first_policy();  // the M-side operand (data matrix / activations)
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
         const int nt = tile % p.n_tiles, j = p.batch - 1 - (tile / p.n_tiles) % p.batch, mt = tile / (p.n_tiles * p.batch);
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
           mbar_expect_tx(s.full[st], tx);
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
-          tma_load_3d(a, &tmA, mt * 128, kc * 64, j, s.full[st]);
-          tma_load_3d(a + 8192, &tmA, mt * 128 + 64, kc * 64, j, s.full[st]);
+          tma_load_3d_hint(a, &tmA, mt * 128, kc * 64, j, s.full[st], stream_once);
+          tma_load_3d_hint(a + 8192, &tmA, mt * 128 + 64, kc * 64, j, s.full[st], stream_once);
           for (int nb = 0; nb < p.nbox; ++nb)
             tma_load_3d(a + kABytes + nb * 8192, &tmB, nt * 256 + nb * 64, kc * 64, j, s.full[st]);
           if (++st == kStages) { st = 0; ph ^= 1u; }
@@ -1126,6 +1129,7 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     if (lane == 0) {
       int st = 0;
       uint32_t ph = 0;
+      const uint64_t stream_once = l2_evict_first_policy();  // the data matrix: read once by this kernel
       for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
         const int nt = tile % p.n_tiles, rb = (tile / p.n_tiles) % p.row_blocks, j = tile / (p.n_tiles * p.row_blocks);
         for (int kc = 0; kc < p.num_k; ++kc) {
@@ -1133,7 +1137,7 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (rank == 0) mbar_expect_tx(s.full[st], 2 * kPairStageBytes);
           const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
           const uint32_t bar = map_to_rank(s.full[st], 0);
-          tma_load_3d_pair(a, &tmX, kc * 64, rb * 256 + (int)rank * 128, j, bar);
+          tma_load_3d_pair_hint(a, &tmX, kc * 64, rb * 256 + (int)rank * 128, j, bar, stream_once);
           tma_load_2d_pair(a + 16384, &tmW, kc * 64, nt * 256 + (int)rank * 128, bar);
           if (++st == kPairStages) { st = 0; ph ^= 1u; }
         }
@@ -1221,6 +1225,7 @@ tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       int st = 0;
       uint32_t ph = 0;
+      const uint64_t stream_once = l2_evict_first_policy();  // the M-side operand: the data matrix
       for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
         const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = p.batch - 1 - tile / (p.n_tiles * p.m_tiles);
         const int m0 = mt * 256 + (int)rank * 128, n0 = nt * 256 + (int)rank * 128;
@@ -1229,10 +1234,11 @@ tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (rank == 0) mbar_expect_tx(s.full[st], 2 * kPairStageBytes);
           const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
           const uint32_t bar = map_to_rank(s.full[st], 0);
-          tma_load_3d_pair(a, &tmA, m0, kc * 64, j, bar);
-          tma_load_3d_pair(a + 8192, &tmA, m0 + 64, kc * 64, j, bar);
-          tma_load_3d_pair(a + 16384, &tmB, n0, kc * 64, j, bar);
-          tma_load_3d_pair(a + 24576, &tmB, n0 + 64, kc * 64, j, bar);
+          tma_load_3d_pair_hint(a, &tmA, m0, kc * 64, j, bar, stream_once);
+          tma_load_3d_pair_hint(a + 8192, &tmA, m0 + 64, kc * 64, j, bar, stream_once);
+          // (the residual of a partition is read by the pairs of its M tiles at about the same time, then never again)
+          tma_load_3d_pair_hint(a + 16384, &tmB, n0, kc * 64, j, bar, stream_once);
+          tma_load_3d_pair_hint(a + 24576, &tmB, n0 + 64, kc * 64, j, bar, stream_once);
           if (++st == kPairStages) { st = 0; ph ^= 1u; }
         }
       }
@@ -1377,6 +1383,7 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       int st = 0;
       uint32_t ph = 0;
+      const uint64_t stream_once = l2_evict_first_policy();  // the N-side operand: the data matrix
       for (int u = pair_id; u < p.num_units && !failed; u += n_pairs) {
         const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
         int w0, w1;
@@ -1390,11 +1397,12 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (rank == 0) mbar_expect_tx(full[st], tx);
           const uint32_t a = smem_u32(tiles + st * kWideStageBytes);
           const uint32_t bar = map_to_rank(full[st], 0);
-          tma_load_3d_pair(a, &tmA, m0, kc * 64, j, bar);
-          tma_load_3d_pair(a + 8192, &tmA, m0 + 64, kc * 64, j, bar);
-          for (int b = 0; b < nb0; ++b) tma_load_3d_pair(a + 16384 + b * 8192, &tmB, c0 + b * 64, kc * 64, j, bar);
+          tma_load_3d_pair_hint(a, &tmA, m0, kc * 64, j, bar, stream_once);
+          tma_load_3d_pair_hint(a + 8192, &tmA, m0 + 64, kc * 64, j, bar, stream_once);
+          for (int b = 0; b < nb0; ++b)
+            tma_load_3d_pair_hint(a + 16384 + b * 8192, &tmB, c0 + b * 64, kc * 64, j, bar, stream_once);
           for (int b = 0; b < nb1; ++b)
-            tma_load_3d_pair(a + 16384 + (nb0 + b) * 8192, &tmB, c1 + b * 64, kc * 64, j, bar);
+            tma_load_3d_pair_hint(a + 16384 + (nb0 + b) * 8192, &tmB, c1 + b * 64, kc * 64, j, bar, stream_once);
           if (++st == kWideStages) { st = 0; ph ^= 1u; }
         }
       }
