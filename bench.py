@@ -454,8 +454,11 @@ def measure_side_workload(name, dev, peaks, which, smi_index, args):
     kern_ms, kern_n = kernel_bracket(pb, pats, min(steps, 50))
     clocks = sampler.stop()
     host_us = host_queue_us(pb, pats, steps)
-    out = {"ms_per_step": med, "ms_per_step_mean_of_queued": total_ms / steps, "steps": steps, "warmup": warm,
-           "gradients_per_s": 1e3 / med,
+    # ms_per_step as in the headline: steps queued back to back between two events.  The median of single steps
+    # has an event between every two steps, which keeps a step's first kernels from being set up under the step
+    # before (programmatic dependent launch) and so reads 5-10 % higher for the short dense steps.
+    out = {"ms_per_step": total_ms / steps, "ms_per_step_median_of_single_steps": med, "steps": steps, "warmup": warm,
+           "gradients_per_s": 1e3 * steps / total_ms,
            "roofline": roofline_of(w, pb.cdt == pb.ngc.NGC_F64, kern_ms, kern_n, peaks, which, TRAFFIC_BYTES.get(name)),
            "clocks": clocks, "host_us_per_step_call": host_us, "prep_ms_once": pb.prep_ms,
            "undecodable_skipped": skipped,
@@ -569,7 +572,7 @@ def run_cuda(args):
         "e2e": e2e,
         "gpu_launches": int(rank_sum(launches, world, dev)),
         "roofline": roofline,
-        "ms_per_step_median": median_ms,
+        "ms_per_step_median_of_single_steps": median_ms,
         "host_us_per_step_call": host_us,
         "prep_ms_once": pb.prep_ms,
         "decode_residual_max": residual,
@@ -585,7 +588,7 @@ def run_cuda(args):
         side = {}
         for name in SIDE_WORKLOADS:
             if name == w.name:
-                side[name] = {"ms_per_step": median_ms if median_ms is not None else ms_total / args.steps,
+                side[name] = {"ms_per_step": ms_total / args.steps, "ms_per_step_median_of_single_steps": median_ms,
                               "roofline": roofline, "clocks": clocks, "parity": line.get("parity"),
                               "see": "top level of this line"}
                 continue

@@ -199,7 +199,7 @@ namespace {
 // Encode of a dense model's partial gradients; with a hook, the decode in the same kernel.
 int encode_dense(ngc_plan_t *p, const ngc::RowSplit &split, const float *G, long long ldG, const ngc_level_t &lv,
                  long long l, void *coded, int cdt, cudaStream_t stream, DecodeHook *hook) {
-  if (!hook) {
+  if (!hook || !hook->grad) {  // no decode to take along (or its vector is not solved before the encode)
     NGC_CUDA(p, ngc::launch_encode_long(split, G, ldG, lv.d_coef, p->n, lv.s, l, coded, cdt, stream));
     return NGC_OK;
   }
@@ -506,6 +506,7 @@ int ngc_step(ngc_plan_t *p, const ngc_model_t *m, const void *theta, const void 
     // The gradient kernel fills its SMs: the solve waits for it on the side stream and runs beside the small
     // encode kernel instead of in line behind it.
     hook.after_grads = static_cast<cudaEvent_t>(p->ev_grads);
+    hook.grad = nullptr;  // the vector is solved after the gradients: the decode stays a kernel of its own
   }
   // Dense models: the encode kernel forms the decoded gradient from the coded rows as it writes them.
   rc = grad_encode_impl(p, m, theta, X, y, info->layer, coded, cuda_stream, &hook);
