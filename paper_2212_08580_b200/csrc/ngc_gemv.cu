@@ -37,6 +37,7 @@ struct GemvParams {
   int row_bytes;
   int stage_bytes;
   int stages;
+  int act;  // 0: residual z - y (least squares), 1: sigmoid(z) - y (logistic)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -102,30 +103,32 @@ struct Vec<__nv_bfloat16> {
   }
 };
 
-// Walks the tiles of one CTA range: at most R rows, never crossing a partition-group boundary.
+// Walks the tiles of one CTA range: at most R rows, never crossing a partition-group boundary.  Positions are
+// kept relative to the first row of the range (32 bits: a range is the 148th part of the data), the absolute
+// 64-bit row index is formed only where an address is.
 struct TileWalk {
-  long long cur, end, seg_end, rows_g;
+  long long base;
+  int cur, end, seg_end, rows_g;
   int group;
   __device__ __forceinline__ void init(long long b, long long e, long long rg) {
-    cur = b; end = e; rows_g = rg;
+    base = b; cur = 0; end = (int)(e - b); rows_g = (int)rg;
     group = (int)(b / rg);
-    seg_end = (long long)(group + 1) * rg;
-    if (seg_end > end) seg_end = end;
+    const long long se = (long long)(group + 1) * rg - b;
+    seg_end = se < (long long)end ? (int)se : end;
   }
   __device__ __forceinline__ bool done() const { return cur >= end; }
   // returns the tile starting at `cur`; seg_last = it closes this CTA's piece of partition group `g`
   __device__ __forceinline__ void next(int R, long long &row0, int &nrows, bool &seg_last, int &g) {
-    long long e = cur + R;
+    int e = cur + R;
     if (e > seg_end) e = seg_end;
-    row0 = cur;
-    nrows = (int)(e - cur);
+    row0 = base + cur;
+    nrows = e - cur;
     g = group;
     seg_last = (e == seg_end);
     cur = e;
     if (seg_last) {
       ++group;
-      seg_end += rows_g;
-      if (seg_end > end) seg_end = end;
+      seg_end = (seg_end > end - rows_g) ? end : seg_end + rows_g;
     }
   }
 };
@@ -159,7 +162,7 @@ template <> struct Log2<2> { static constexpr int v = 1; };
 template <> struct Log2<4> { static constexpr int v = 2; };
 template <> struct Log2<8> { static constexpr int v = 3; };
 
-template <typename XT, int VPT, int R, int ACT>
+template <typename XT, int VPT, int R>
 __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams p) {
   pdl_sync();
   constexpr int VN = Vec<XT>::N;
@@ -264,9 +267,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
 #pragma unroll
       for (int off = kWarps / 2; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
       if (lane == 0) {
-        float res;
-        if (ACT == 1) res = 1.f / (1.f + expf(-z)) - yrow;
-        else res = z - yrow;
+        // (one code path for both activations: as two template instances the least-squares one, although the
+        // simpler, was compiled with spills at the 128-register cap of the widest bf16 shape)
+        const float res = (p.act ? 1.f / (1.f + expf(-z)) : z) - yrow;
         resv[warp] = (warp < nrows) ? res : 0.f;
       }
     }
@@ -320,10 +323,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
   }
 }
 
-template <typename XT, int VPT, int R, int ACT>
+template <typename XT, int VPT, int R>
 cudaError_t launch_one(const GemvParams &p, cudaStream_t stream) {
   const size_t smem = (size_t)p.stages * p.stage_bytes + kSmemReserve;
-  auto kern = gemv_pair_kernel<XT, VPT, R, ACT>;
+  auto kern = gemv_pair_kernel<XT, VPT, R>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   launch_k(kern, p.split.grid, kThreads, smem, stream, p);
@@ -332,15 +335,15 @@ cudaError_t launch_one(const GemvParams &p, cudaStream_t stream) {
 
 // Whether one more small block (a warp or two, a few KB of shared memory) still fits on an SM that
 // holds a CTA of this kernel: registers are what runs out first (512 threads x 128 registers fill the file).
-template <typename XT, int VPT, int R, int ACT>
+template <typename XT, int VPT, int R>
 bool room_beside(const GemvParams &p) {
   cudaFuncAttributes attr;
-  if (cudaFuncGetAttributes(&attr, gemv_pair_kernel<XT, VPT, R, ACT>) != cudaSuccess) return false;
+  if (cudaFuncGetAttributes(&attr, gemv_pair_kernel<XT, VPT, R>) != cudaSuccess) return false;
   const size_t smem = (size_t)p.stages * p.stage_bytes + kSmemReserve;
   return (size_t)attr.numRegs * kThreads + 64 * 64 <= 65536 && smem + 16384 <= 233472;
 }
 
-template <typename XT, int ACT>
+template <typename XT>
 cudaError_t launch_shape(GemvParams &p, cudaStream_t stream, bool *room = nullptr) {
   const int nv = p.d / Vec<XT>::N;
   int vpt = (nv + kThreads - 1) / kThreads;
@@ -355,12 +358,12 @@ cudaError_t launch_shape(GemvParams &p, cudaStream_t stream, bool *room = nullpt
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
   if (room) {  // query only, nothing is launched
-    *room = (vpt == 1) ? room_beside<XT, 1, 8, ACT>(p) : (vpt == 2) ? room_beside<XT, 2, 4, ACT>(p) : room_beside<XT, 4, 2, ACT>(p);
+    *room = (vpt == 1) ? room_beside<XT, 1, 8>(p) : (vpt == 2) ? room_beside<XT, 2, 4>(p) : room_beside<XT, 4, 2>(p);
     return cudaSuccess;
   }
-  if (vpt == 1) return launch_one<XT, 1, 8, ACT>(p, stream);
-  if (vpt == 2) return launch_one<XT, 2, 4, ACT>(p, stream);
-  return launch_one<XT, 4, 2, ACT>(p, stream);
+  if (vpt == 1) return launch_one<XT, 1, 8>(p, stream);
+  if (vpt == 2) return launch_one<XT, 2, 4>(p, stream);
+  return launch_one<XT, 4, 2>(p, stream);
 }
 
 }  // namespace
@@ -389,24 +392,22 @@ cudaError_t launch_gemv_pair(const ngc_model_t &m, const RowSplit &split, const 
   p.status = status;
   p.split = split;
   p.d = m.d;
-  const int act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
+  p.act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
   if (m.x_dtype == NGC_F32) {
     p.row_bytes = m.d * 4;
-    return act ? launch_shape<float, 1>(p, stream) : launch_shape<float, 0>(p, stream);
+    return launch_shape<float>(p, stream);
   }
   p.row_bytes = m.d * 2;
-  return act ? launch_shape<__nv_bfloat16, 1>(p, stream) : launch_shape<__nv_bfloat16, 0>(p, stream);
+  return launch_shape<__nv_bfloat16>(p, stream);
 }
 
 bool gemv_pair_leaves_room(const ngc_model_t &m) {
   GemvParams p;
   p.d = m.d;
   p.row_bytes = m.d * (m.x_dtype == NGC_F32 ? 4 : 2);
-  const int act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
+  p.act = (m.kind == NGC_LOGISTIC) ? 1 : 0;
   bool room = false;
-  cudaError_t e;
-  if (m.x_dtype == NGC_F32) e = act ? launch_shape<float, 1>(p, 0, &room) : launch_shape<float, 0>(p, 0, &room);
-  else e = act ? launch_shape<__nv_bfloat16, 1>(p, 0, &room) : launch_shape<__nv_bfloat16, 0>(p, 0, &room);
+  const cudaError_t e = (m.x_dtype == NGC_F32) ? launch_shape<float>(p, 0, &room) : launch_shape<__nv_bfloat16>(p, 0, &room);
   return e == cudaSuccess && room;
 }
 
