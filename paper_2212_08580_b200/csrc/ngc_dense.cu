@@ -71,9 +71,16 @@ struct TnParams {
   int *status;
 };
 
+// Consecutive mbarriers addressed by index: the address is computed, not looked up (an array of addresses indexed by
+// a run-time stage number would live in local memory and cost a load on every wait of the issuing threads).
+struct BarArray {
+  uint32_t base;
+  __device__ __forceinline__ uint32_t operator[](int i) const { return base + 8u * (uint32_t)i; }
+};
+
 struct Smem {
   unsigned char *tiles;
-  uint32_t full[kStages], empty[kStages], tfull[2], tempty[2];
+  BarArray full, empty, tfull, tempty;
   uint32_t *tmem_slot;
   volatile int *abort_flag;
   float *xch;
@@ -87,14 +94,10 @@ __device__ __forceinline__ Smem carve(unsigned char *raw, int nst) {
   s.tiles = raw + ((1024u - (base & 1023u)) & 1023u);
   s.nst = nst;
   uint64_t *bars = reinterpret_cast<uint64_t *>(s.tiles + nst * kStageBytes);
-  for (int i = 0; i < kStages; ++i) {
-    s.full[i] = smem_u32(&bars[i]);
-    s.empty[i] = smem_u32(&bars[kStages + i]);
-  }
-  s.tfull[0] = smem_u32(&bars[2 * kStages]);
-  s.tfull[1] = smem_u32(&bars[2 * kStages + 1]);
-  s.tempty[0] = smem_u32(&bars[2 * kStages + 2]);
-  s.tempty[1] = smem_u32(&bars[2 * kStages + 3]);
+  s.full.base = smem_u32(&bars[0]);
+  s.empty.base = smem_u32(&bars[kStages]);
+  s.tfull.base = smem_u32(&bars[2 * kStages]);
+  s.tempty.base = smem_u32(&bars[2 * kStages + 2]);
   s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kStages + 4]);
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
   s.xch = reinterpret_cast<float *>(s.tiles + nst * kStageBytes + 256);
@@ -629,13 +632,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   // The tile lives in shared memory as groups of two 64-column chunks.  Group g is loaded (h), consumed,
   // overwritten in place (delta1), stored and reloaded with the next tile's h on its own barriers, so the
   // memory traffic of the finished groups hides behind the arithmetic on the others.
-  uint32_t h_full[4], m_done[4], w_done[4];
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    h_full[g] = smem_u32(&bars[g]);
-    m_done[g] = smem_u32(&bars[4 + g]);
-    w_done[g] = smem_u32(&bars[8 + g]);
-  }
+  const BarArray h_full{smem_u32(&bars[0])}, m_done{smem_u32(&bars[4])}, w_done{smem_u32(&bars[8])};
   const uint32_t z_full = smem_u32(&bars[12]), d2_full = smem_u32(&bars[13]), d_full = smem_u32(&bars[14]),
                  d_empty = smem_u32(&bars[15]), w_full = smem_u32(&bars[16]);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[17]);
@@ -1056,7 +1053,7 @@ constexpr int kSmemPair = kPairStages * kPairStageBytes + 1024 + 256 + kXchBytes
 
 struct PairSmem {
   unsigned char *tiles;
-  uint32_t full[kPairStages], empty[kPairStages], tfull[2], tempty[2];
+  BarArray full, empty, tfull, tempty;
   uint32_t *tmem_slot;
   volatile int *abort_flag;
   float *xch;
@@ -1068,14 +1065,10 @@ __device__ __forceinline__ PairSmem carve_pair(unsigned char *raw) {
   const uint32_t base = smem_u32(raw);
   s.tiles = raw + ((1024u - (base & 1023u)) & 1023u);
   uint64_t *bars = reinterpret_cast<uint64_t *>(s.tiles + kPairStages * kPairStageBytes);
-  for (int i = 0; i < kPairStages; ++i) {
-    s.full[i] = smem_u32(&bars[i]);
-    s.empty[i] = smem_u32(&bars[kPairStages + i]);
-  }
-  s.tfull[0] = smem_u32(&bars[2 * kPairStages]);
-  s.tfull[1] = smem_u32(&bars[2 * kPairStages + 1]);
-  s.tempty[0] = smem_u32(&bars[2 * kPairStages + 2]);
-  s.tempty[1] = smem_u32(&bars[2 * kPairStages + 3]);
+  s.full.base = smem_u32(&bars[0]);
+  s.empty.base = smem_u32(&bars[kPairStages]);
+  s.tfull.base = smem_u32(&bars[2 * kPairStages]);
+  s.tempty.base = smem_u32(&bars[2 * kPairStages + 2]);
   s.tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kPairStages + 4]);
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
   s.xch = reinterpret_cast<float *>(s.tiles + kPairStages * kPairStageBytes + 256);
@@ -1350,12 +1343,7 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t sbase = smem_u32(smem_raw);
   unsigned char *tiles = smem_raw + ((1024u - (sbase & 1023u)) & 1023u);
   uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + kWideStages * kWideStageBytes);
-  uint32_t full[kWideStages], empty[kWideStages];
-#pragma unroll
-  for (int i = 0; i < kWideStages; ++i) {
-    full[i] = smem_u32(&bars[i]);
-    empty[i] = smem_u32(&bars[kWideStages + i]);
-  }
+  const BarArray full{smem_u32(&bars[0])}, empty{smem_u32(&bars[kWideStages])};
   const uint32_t tfull = smem_u32(&bars[2 * kWideStages]), tempty = smem_u32(&bars[2 * kWideStages + 1]);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kWideStages + 2]);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
