@@ -498,7 +498,8 @@ encode_window_kernel(const float *__restrict__ ws, long long ld_ws, const double
                      long long d, int chunk, CT *__restrict__ coded, const double *__restrict__ avec,
                      double *__restrict__ gpart, float *__restrict__ grad) {
   pdl_sync();
-  constexpr int W = S1 + kEncLook;
+  // wide windows keep fewer loads in flight: the ring is what fills the registers (measured at S1 = 11: 3 better than 6)
+  constexpr int W = S1 + (S1 >= 8 ? 3 : kEncLook);
   __shared__ CT cs[NGC_MAX_N * S1];
   __shared__ double as[DEC ? NGC_MAX_N : 1];
   const int first = blockIdx.y * chunk;
