@@ -560,7 +560,8 @@ def run_cuda(args):
         "config": {"workload": w.name, "n_workers": w.n, "levels": list(w.levels), "kind": w.kind,
                    "rows_per_partition": w.rows, "d": w.d, "x_dtype": w.x_dtype,
                    "coded_dtype": "f64" if pb.cdt == pb.ngc.NGC_F64 else "f32",
-                   "l2": "inputs larger than L2 (data matrix %.2f GB per step)" % (h2d / 1e9),
+                   "l2": ("inputs larger than L2 (data matrix %.2f GB per step)" % (h2d / 1e9)) if h2d > 126e6 else
+                         "inputs fit in L2: a latency figure, no roofline claim",
                    "patterns": "fresh seeded pattern per step", "undecodable_skipped": skipped,
                    "levels_chosen": {str(k): levels_used.count(k) for k in sorted(set(levels_used))},
                    "replicas": "independent per GPU, no data-path collective",
