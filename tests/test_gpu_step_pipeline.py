@@ -125,3 +125,32 @@ def test_dense_steps_are_bitwise_reproducible(name, rows):
         outs.append((coded.cpu(), grad.cpu()))
     for c, g in outs[1:]:
         assert torch.equal(c, outs[0][0]) and torch.equal(g, outs[0][1])
+
+
+@pytest.mark.parametrize("name,rows,tol", [("lsq100", 64, 1e-5), ("mlp30", 200, 1e-2)])
+def test_step_from_host_buffers_matches_the_device_step(name, rows, tol):
+    """ngc_step_host (host buffers in, host gradient out: the end-to-end entry point the benchmark times) gives the
+    bits of ngc_step on device copies of the same buffers, also while another data matrix is prepared on the plan."""
+    from dataclasses import replace
+    w = replace(ngc_inputs.shrink(ngc_inputs.WORKLOADS[name], rows=rows), pattern="sets")
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    l = w.n_params
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    cdt = torch.float64 if p.coded_dtype(m) == ngc.NGC_F64 else torch.float32
+    coded = torch.empty((w.n, l), dtype=cdt, device="cuda")
+    grad = torch.empty(l, dtype=torch.float32, device="cuda")
+    p.prepare_data(m, X)                                    # the host path must not pick this copy up for other data
+    Xh = (X.float() * 0.5).to(X.dtype).cpu().pin_memory()   # other contents than the prepared matrix
+    yh, thh = y.cpu().pin_memory(), theta.cpu().pin_memory()
+    gh = torch.empty(l, dtype=torch.float32).pin_memory()
+    for stragglers in ([], [2], list(range(w.levels[-1]))):
+        t = ngc_inputs.set_times(w.n, w.levels[-1] + 1, stragglers)
+        info_h = p.step_host(m, thh, Xh, yh, t, gh)
+        info_d = p.step(m, theta, Xh.cuda(), y, t, coded, grad)
+        torch.cuda.synchronize()
+        assert info_h.layer == info_d.layer and list(info_h.responsive()) == list(info_d.responsive())
+        assert torch.equal(gh, grad.cpu())
+        G = oracle_G(w, Xh.cuda(), y, theta)
+        assert rel_l2(gh.numpy(), G.sum(axis=0)) < tol
+    assert p.device_status() < 1e-6
