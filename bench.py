@@ -410,6 +410,32 @@ def host_queue_us(pb, pats, steps):
     return 1e6 * dt / steps
 
 
+def grad_encode_per_level(pb, peaks, launches=20):
+    """ngc_grad_encode (gradient kernels + encode, no selection, no decode) timed level by level: `launches` calls
+    queued between two events after three untimed ones.  `achieved` divides the same algorithmic bytes / flops as
+    the roofline object by this time, which here includes the encode kernel."""
+    torch, w = pb.torch, pb.w
+    hbm = w.kind in ("lsq", "logistic")
+    work = algorithmic_bytes(w, 8 if pb.cdt == pb.ngc.NGC_F64 else 4) if hbm else algorithmic_flops(w)
+    peak = peaks["hbm_gbs"] if hbm else peaks.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS_SUSTAINED)
+    out = []
+    for layer, s in enumerate(w.levels):
+        for _ in range(3):
+            pb.plan.grad_encode(pb.m, pb.theta, pb.X, pb.y, layer, pb.coded, pb.stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(launches):
+            pb.plan.grad_encode(pb.m, pb.theta, pb.X, pb.y, layer, pb.coded, pb.stream)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / launches
+        achieved = work / (ms * 1e-3) / (1e9 if hbm else 1e12)
+        out.append({"s": s, "ms": ms, "achieved": achieved, "unit": "GB/s" if hbm else "TFLOP/s",
+                    "frac": achieved / peak})
+    return out
+
+
 def cpu_baseline_and_parity(pb, pats, budget_s):
     """The oracle, as it stands, timed on the host cores on a reduced copy of the workload; the library then runs
     the same reduced problem, which gives the parity figure of this very run."""
@@ -454,12 +480,14 @@ def measure_side_workload(name, dev, peaks, which, smi_index, args):
     kern_ms, kern_n = kernel_bracket(pb, pats, min(steps, 50))
     clocks = sampler.stop()
     host_us = host_queue_us(pb, pats, steps)
+    per_level = grad_encode_per_level(pb, peaks)
     # ms_per_step as in the headline: steps queued back to back between two events.  The median of single steps
     # has an event between every two steps, which keeps a step's first kernels from being set up under the step
     # before (programmatic dependent launch) and so reads 5-10 % higher for the short dense steps.
     out = {"ms_per_step": total_ms / steps, "ms_per_step_median_of_single_steps": med, "steps": steps, "warmup": warm,
            "gradients_per_s": 1e3 * steps / total_ms,
            "roofline": roofline_of(w, pb.cdt == pb.ngc.NGC_F64, kern_ms, kern_n, peaks, which, TRAFFIC_BYTES.get(name)),
+           "grad_encode_per_level": per_level,
            "clocks": clocks, "host_us_per_step_call": host_us, "prep_ms_once": pb.prep_ms,
            "undecodable_skipped": skipped,
            "levels_chosen": {str(k): levels.count(k) for k in sorted(set(levels))},
@@ -523,6 +551,8 @@ def run_cuda(args):
     kern_ms, kern_n = kernel_bracket(pb, pats[args.warmup:], min(max(args.steps, 20), 100))
     clocks = sampler.stop() if rank == 0 else {}
     host_us = host_queue_us(pb, pats[args.warmup:], min(max(args.steps, 20), 200))
+    peaks, which = measured_peaks()
+    per_level = grad_encode_per_level(pb, peaks) if rank == 0 and world == 1 else None
     residual = pb.plan.device_status()
 
     # ---- end to end through the host-buffer entry point: pinned host inputs copied every step
@@ -548,7 +578,6 @@ def run_cuda(args):
                "d2h_bytes_per_step": d2h, "steps": e2e_steps}
         del Xh, yh, thh, gh
 
-    peaks, which = measured_peaks()
     traffic = TRAFFIC_BYTES.get(w.name) if not args.rows else None
     roofline = roofline_of(w, pb.cdt == pb.ngc.NGC_F64, kern_ms, kern_n, peaks, which, traffic)
 
@@ -573,6 +602,7 @@ def run_cuda(args):
         "e2e": e2e,
         "gpu_launches": int(rank_sum(launches, world, dev)),
         "roofline": roofline,
+        "grad_encode_per_level": per_level,
         "ms_per_step_median_of_single_steps": median_ms,
         "host_us_per_step_call": host_us,
         "prep_ms_once": pb.prep_ms,
@@ -590,7 +620,8 @@ def run_cuda(args):
         for name in SIDE_WORKLOADS:
             if name == w.name:
                 side[name] = {"ms_per_step": ms_total / args.steps, "ms_per_step_median_of_single_steps": median_ms,
-                              "roofline": roofline, "clocks": clocks, "parity": line.get("parity"),
+                              "roofline": roofline, "grad_encode_per_level": per_level, "clocks": clocks,
+                              "parity": line.get("parity"),
                               "see": "top level of this line"}
                 continue
             side[name] = measure_side_workload(name, dev, peaks, which, smi_index, args)
