@@ -313,6 +313,22 @@ int ngc_device_status(ngc_plan_t *plan, double *residual_out);
  * plan and the CUDA context remain usable.  Nothing faults or hangs.
  */
 int ngc_selftest_wait_timeout(ngc_plan_t *plan, int64_t limit_cycles, void *cuda_stream);
+/*
+ * Introspection for tests (host only, no GPU needed; a property of the library, the paper has no
+ * counterpart).  The backward contractions of the dense models on CTA pairs (softmax: G_j = X_j^T R_j with the
+ * 256 classes on the M side; MLP: [dW1; db1] = [X 1]^T delta1 with the hidden units on the M side in
+ * `m_blocks` blocks of 256) cut the `n_cols` columns of the other operand into passes of 512 columns, may
+ * cut some passes into halves of 256 to even out the load, and deal these units to at most `max_pairs`
+ * CTA pairs.  This call returns that unit list for a problem of `batch` partitions and `k_chunks` chunks of
+ * 64 rows per partition: row u of units_out (caller-owned host array of cap rows x 8 int32) gets
+ * {pair, round, partition, M block, first column, width, first column, width} of the u-th unit in the order
+ * the pairs take them; a second width of 0 means the unit has one column range.  Widths are multiples of
+ * 32 and at most 256; ranges may run past n_cols (those columns are neither read nor stored).
+ * *n_units_out gets the number of units (which may exceed cap: then only cap rows were written),
+ * *n_pairs_out the number of pairs.  NGC_ERR_INVALID for non-positive sizes or NULL outputs.
+ */
+int ngc_dense_schedule(int batch, int m_blocks, int n_cols, int k_chunks, int max_pairs, int32_t *units_out, int cap,
+                       int *n_units_out, int *n_pairs_out);
 /* cudaError_t of the last failed runtime call on this plan (0 if none). */
 int ngc_last_cuda_error(const ngc_plan_t *plan);
 /* How many kernels of this library the plan has launched so far. */

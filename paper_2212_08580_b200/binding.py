@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
         "ngc_gd_update": (i32, [vp, vp, i64, C.c_float, vp]),
         "ngc_sample_times": (i32, [u64, i32, i32, dbl, dbl, dbl, P(dbl)]),
         "ngc_selftest_wait_timeout": (i32, [vp, i64, vp]),
+        "ngc_dense_schedule": (i32, [i32, i32, i32, i32, i32, vp, i32, P(i32), P(i32)]),
         "ngc_profile_enable": (i32, [vp, i32]),
         "ngc_profile_read": (i32, [vp, P(dbl), P(i64)]),
         "ngc_workspace_bytes": (C.c_size_t, [vp]),
@@ -121,6 +122,22 @@ def sample_times(seed: int, n: int, tasks: int, shift: float, rate: float, p_fai
     if rc != 0:
         raise NgcError(rc, "ngc_sample_times")
     return out
+
+
+def dense_schedule(batch: int, m_blocks: int, n_cols: int, k_chunks: int, max_pairs: int):
+    """ngc_dense_schedule: (units [n][8] int32 = pair, round, partition, M block, c0, w0, c1, w1; number of pairs)."""
+    lib = load_library()
+    n_units, n_pairs = C.c_int32(0), C.c_int32(0)
+    rc = lib.ngc_dense_schedule(batch, m_blocks, n_cols, k_chunks, max_pairs, None, 0, C.byref(n_units),
+                                C.byref(n_pairs))
+    if rc != 0:
+        raise NgcError(rc, "ngc_dense_schedule")
+    units = np.empty((n_units.value, 8), dtype=np.int32)
+    rc = lib.ngc_dense_schedule(batch, m_blocks, n_cols, k_chunks, max_pairs, units.ctypes.data_as(C.c_void_p),
+                                units.shape[0], C.byref(n_units), C.byref(n_pairs))
+    if rc != 0:
+        raise NgcError(rc, "ngc_dense_schedule")
+    return units, n_pairs.value
 
 
 def latency_cdf_gc(n, sigma, t, lam, rho, gamma, eps, p_fail) -> float:

@@ -603,6 +603,17 @@ int ngc_selftest_wait_timeout(ngc_plan_t *p, int64_t limit_cycles, void *cuda_st
   return NGC_OK;
 }
 
+int ngc_dense_schedule(int batch, int m_blocks, int n_cols, int k_chunks, int max_pairs, int32_t *units_out, int cap,
+                       int *n_units_out, int *n_pairs_out) {
+  if (batch < 1 || m_blocks < 1 || n_cols < 1 || k_chunks < 1 || max_pairs < 1 || cap < 0 || !n_units_out ||
+      !n_pairs_out || (cap > 0 && !units_out))
+    return NGC_ERR_INVALID;
+  static_assert(sizeof(int32_t) == sizeof(int), "unit rows are written as int");
+  *n_units_out = ngc::wide_schedule_units(batch, m_blocks, n_cols, k_chunks, max_pairs,
+                                          reinterpret_cast<int *>(units_out), cap, n_pairs_out);
+  return NGC_OK;
+}
+
 int ngc_profile_enable(ngc_plan_t *p, int on) {
   if (!p) return NGC_ERR_INVALID;
   p->profiling = on != 0;

@@ -1202,121 +1202,43 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   pair_teardown(warp, tmem_base, failed, p.status);
 }
 
-// Backward contraction on a CTA pair: tile = (batch j, 256 rows of M, 256 columns of N); N must be 256.
-__global__ void __launch_bounds__(kTcThreads, 1)
-tn_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TnParams p) {
-  pdl_sync();
-  extern __shared__ unsigned char smem_raw[];
-  const PairSmem s = carve_pair(smem_raw);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_rank();
-  const uint32_t tmem_base = pair_prologue(s, warp, kTcThreads - 64);
-  bool failed = false;
-  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      int st = 0;
-      uint32_t ph = 0;
-      const uint64_t stream_once = l2_evict_first_policy();  // the M-side operand: the data matrix
-      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
-        const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = p.batch - 1 - tile / (p.n_tiles * p.m_tiles);
-        const int m0 = mt * 256 + (int)rank * 128, n0 = nt * 256 + (int)rank * 128;
-        for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(s.empty[st], ph ^ 1u)) { failed = true; break; }
-          if (rank == 0) mbar_expect_tx(s.full[st], 2 * kPairStageBytes);
-          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
-          const uint32_t bar = map_to_rank(s.full[st], 0);
-          tma_load_3d_pair_hint(a, &tmA, m0, kc * 64, j, bar, stream_once);
-          tma_load_3d_pair_hint(a + 8192, &tmA, m0 + 64, kc * 64, j, bar, stream_once);
-          // (the residual of a partition is read by the pairs of its M tiles at about the same time, then never again)
-          tma_load_3d_pair_hint(a + 16384, &tmB, n0, kc * 64, j, bar, stream_once);
-          tma_load_3d_pair_hint(a + 24576, &tmB, n0 + 64, kc * 64, j, bar, stream_once);
-          if (++st == kPairStages) { st = 0; ph ^= 1u; }
-        }
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
-      const uint32_t idesc = instr_desc_bf16(256, 256, 1, 1);
-      int st = 0, buf = 0;
-      uint32_t ph = 0, aph = 0;
-      for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
-        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
-        tc_fence_after();
-        const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
-        for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
-          tc_fence_after();
-          const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
-          const uint64_t ad = smem_desc_sw128(a, 8192, 1024), bd = smem_desc_sw128(a + 16384, 8192, 1024);
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            mma_bf16_pair(acc, ad + (uint64_t)(k4 * 128), bd + (uint64_t)(k4 * 128), idesc, (kc | k4) != 0);
-          mma_commit_pair(s.empty[st], 3);
-          if (++st == kPairStages) { st = 0; ph ^= 1u; }
-        }
-        if (failed) break;
-        mma_commit_pair(s.tfull[buf], 3);
-        buf ^= 1;
-        if (buf == 0) aph ^= 1u;
-      }
-    }
-  } else {
-    const int q = warp & 3;
-    int buf = 0;
-    uint32_t aph = 0;
-    const bool vec = (p.out_ld % 4 == 0) && (p.out_batch % 4 == 0);
-    for (int tile = pair_id; tile < p.num_tiles; tile += n_pairs) {
-      const int nt = tile % p.n_tiles, mt = (tile / p.n_tiles) % p.m_tiles, j = p.batch - 1 - tile / (p.n_tiles * p.m_tiles);
-      if (!mbar_wait(s.tfull[buf], aph)) { failed = true; break; }
-      tc_fence_after();
-      const int m = mt * 256 + (int)rank * 128 + q * 32 + lane;
-      const bool valid = m < p.m_store;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
-      float *dst = p.out + (size_t)j * p.out_batch + (size_t)(valid ? m : 0) * p.out_ld + (size_t)nt * 256;
-      float v[32];
-      for (int c0 = 0; c0 < 256; c0 += 32) {
-        tmem_ld32(taddr + c0, v);
-        if (valid) {
-          if (vec) {
-#pragma unroll
-            for (int g4 = 0; g4 < 8; ++g4)
-              *reinterpret_cast<float4 *>(dst + c0 + g4 * 4) = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) dst[c0 + i] = v[i];
-          }
-        }
-      }
-      tc_fence_before();
-      mbar_arrive_cluster(map_to_rank(s.tempty[buf], 0));
-      buf ^= 1;
-      if (buf == 0) aph ^= 1u;
-    }
-  }
-  pair_teardown(warp, tmem_base, failed, p.status);
-}
-
 // ------------------------------------------------------------------------------------------------
 // Wide backward contraction on a CTA pair, roles swapped: D^T = A^T B with A [batch][K][M] on the M side in
 // blocks of 256 (128 per CTA) and B [batch][K][n_total] on the N side in passes of up to 512 columns, so that
 // one pass fills all of tensor memory (two accumulators of up to 256 columns) and the A block is fetched once
 // per 512 columns of B instead of once per 256.  These kernels run at the rate shared memory is fed from L2,
-// not at the tensor cores' rate: a pass moves 96 KB per K chunk for 256 x 512 outputs where two 256 x 256
-// tiles move 128 KB.  A ragged last pass issues a narrower second instruction (N a multiple of 32) instead of
-// a whole padded tile.  D^T(m, n) is stored at out[n * out_ld + m]: consecutive lanes hold consecutive m, so
-// every column of the accumulator leaves as one 128-byte warp store.
-// Unit = (batch j, M block mt, pass p), mt fastest (neighbouring pairs share B through L2), batches last to
-// first (the kernel before went first to last).  Units go round-robin to the pairs.
+// not at the tensor cores' rate: a whole pass moves 96 KB per K chunk for 256 x 512 outputs where two
+// 256 x 256 tiles move 128 KB.  A ragged last pass issues a narrower second instruction (N a multiple of 32)
+// instead of a whole padded tile.  D^T(m, n) is stored at out[n * out_ld + m]: consecutive lanes hold
+// consecutive m, so every column of the accumulator leaves as one 128-byte warp store.
+//
+// Units.  Whole passes keep the traffic low but come in few, long units; so the host may cut some of the
+// whole passes into their two halves of 256 columns (each a unit that uses one accumulator) where that
+// evens out the pairs' loads (wide_schedule).  Units are listed longest first -- whole passes, then the ragged
+// passes and the halves in the order of their cost -- and dealt to the pairs in rounds that alternate
+// direction, so the pair that got the longest unit of one round gets the shortest of the next.  Within
+// a class the order is batch (last to first: the kernel before went first to last), pass, M block, with
+// the M block fastest (neighbouring pairs share B through L2).  A unit that needs one accumulator takes
+// the two accumulators in turn, so its epilogue overlaps the next unit's contraction; after a whole pass
+// the next unit starts as soon as the accumulator it needs has been read out.
 // ------------------------------------------------------------------------------------------------
 constexpr int kWideStages = 4;
 constexpr int kWideStageBytes = 16384 + 4 * 8192;  // 128 x 64 of A + up to four 64 x 64 boxes of B per CTA
 constexpr int kSmemWide = kWideStages * kWideStageBytes + 1024 + 256;
 constexpr int kWideThreads = 320;  // producer, MMA, 8 epilogue warps
 
+struct WideSchedule {
+  int full_passes;   // whole passes of 512 columns per (batch, M block): n_total / 512
+  int n_whole;       // whole passes kept as one unit (the first n_whole in batch / pass / M block order)
+  int n_ragged;      // ragged last passes: batch * m_tiles, or 0
+  int n_half;        // halves of the whole passes that were cut: 2 * (batch * m_tiles * full_passes - n_whole)
+  int ragged_first;  // the ragged passes are dealt before the halves (they cost more)
+  int num_units, pairs;
+};
+
 struct TnWideParams {
-  int batch, m_tiles, n_passes, num_units;
+  int batch, m_tiles;
+  WideSchedule sch;
   int num_k;      // K chunks of 64
   int n_total;    // columns of B that exist in D^T (rows of the stored matrix)
   float *out;     // D^T(j, m, n) -> out[j * out_batch + n * out_ld + m]
@@ -1335,6 +1257,44 @@ __host__ __device__ inline void wide_pass_widths(int n_total, int pass, int *w0,
   *w1 = r1 <= 0 ? 0 : (r1 < 256 ? r1 : 256);
 }
 
+// Unit u of the list: batch j, M block mt, and up to two column ranges [c, c + w) of B (w1 = 0: one range,
+// one accumulator).
+struct WideUnit {
+  int j, mt, c0, w0, c1, w1;
+};
+__host__ __device__ inline WideUnit wide_unit(int batch, int m_tiles, int n_total, const WideSchedule &s, int u) {
+  const int start_ragged = s.ragged_first ? s.n_whole : s.n_whole + s.n_half;
+  const int start_half = s.ragged_first ? s.n_whole + s.n_ragged : s.n_whole;
+  int jr, mt, pass, half = -1;
+  if (u >= start_ragged && u < start_ragged + s.n_ragged) {
+    const int r = u - start_ragged;
+    jr = r / m_tiles; mt = r % m_tiles; pass = s.full_passes;
+  } else {
+    int f = u;
+    if (u >= s.n_whole) {
+      const int v = u - start_half;
+      f = s.n_whole + (v >> 1);
+      half = v & 1;
+    }
+    const int per_batch = m_tiles * s.full_passes;
+    jr = f / per_batch; mt = (f % per_batch) % m_tiles; pass = (f % per_batch) / m_tiles;
+  }
+  WideUnit q;
+  q.j = batch - 1 - jr; q.mt = mt;
+  wide_pass_widths(n_total, pass, &q.w0, &q.w1);
+  q.c0 = pass * 512; q.c1 = q.c0 + 256;
+  if (half == 0) {
+    q.w1 = 0;
+  } else if (half == 1) {
+    q.c0 = q.c1; q.w0 = q.w1; q.w1 = 0;
+  }
+  return q;
+}
+// The i-th unit of pair `pair` (rounds alternate direction); >= num_units: none in this round.
+__host__ __device__ inline int wide_unit_of(int round, int pair, int pairs) {
+  return round * pairs + ((round & 1) ? pairs - 1 - pair : pair);
+}
+
 __global__ void __launch_bounds__(kWideThreads, 1)
 tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const TnWideParams p) {
@@ -1344,8 +1304,8 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   unsigned char *tiles = smem_raw + ((1024u - (sbase & 1023u)) & 1023u);
   uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + kWideStages * kWideStageBytes);
   const BarArray full{smem_u32(&bars[0])}, empty{smem_u32(&bars[kWideStages])};
-  const uint32_t tfull = smem_u32(&bars[2 * kWideStages]), tempty = smem_u32(&bars[2 * kWideStages + 1]);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kWideStages + 2]);
+  const BarArray tfull{smem_u32(&bars[2 * kWideStages])}, tempty{smem_u32(&bars[2 * kWideStages + 2])};  // per accumulator
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[2 * kWideStages + 4]);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
   if (threadIdx.x == 0) {
@@ -1353,8 +1313,10 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       mbar_init(full[i], 1);
       mbar_init(empty[i], 1);
     }
-    mbar_init(tfull, 1);
-    mbar_init(tempty, 2 * (kWideThreads - 64));
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(tfull[i], 1);
+      mbar_init(tempty[i], 2 * (kWideThreads - 64));
+    }
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
@@ -1365,47 +1327,51 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t tmem_base = *tmem_slot;
   bool failed = false;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int per_batch = p.m_tiles * p.n_passes;
+  const int rounds = (p.sch.num_units + n_pairs - 1) / n_pairs;
 
   if (warp == 0) {
     if (lane == 0) {
       int st = 0;
       uint32_t ph = 0;
-      const uint64_t stream_once = l2_evict_first_policy();  // the N-side operand: the data matrix
-      for (int u = pair_id; u < p.num_units && !failed; u += n_pairs) {
-        const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
-        int w0, w1;
-        wide_pass_widths(p.n_total, pass, &w0, &w1);
-        const int nb0 = (w0 / 2 + 63) / 64, nb1 = (w1 / 2 + 63) / 64;  // 64-column boxes of B this CTA loads
-        const int m0 = mt * 256 + (int)rank * 128;
-        const int c0 = pass * 512 + (int)rank * (w0 / 2), c1 = pass * 512 + 256 + (int)rank * (w1 / 2);
+      const uint64_t stream_once = l2_evict_first_policy();  // both operands are read once by this kernel
+      for (int r = 0; r < rounds && !failed; ++r) {
+        const int u = wide_unit_of(r, pair_id, n_pairs);
+        if (u >= p.sch.num_units) continue;
+        const WideUnit q = wide_unit(p.batch, p.m_tiles, p.n_total, p.sch, u);
+        const int nb0 = (q.w0 / 2 + 63) / 64, nb1 = (q.w1 / 2 + 63) / 64;  // 64-column boxes of B this CTA loads
+        const int m0 = q.mt * 256 + (int)rank * 128;
+        const int c0 = q.c0 + (int)rank * (q.w0 / 2), c1 = q.c1 + (int)rank * (q.w1 / 2);
         const uint32_t tx = 2u * (16384u + (uint32_t)(nb0 + nb1) * 8192u);  // both CTAs signal the leader's barrier
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(empty[st], ph ^ 1u)) { failed = true; break; }
           if (rank == 0) mbar_expect_tx(full[st], tx);
           const uint32_t a = smem_u32(tiles + st * kWideStageBytes);
           const uint32_t bar = map_to_rank(full[st], 0);
-          tma_load_3d_pair_hint(a, &tmA, m0, kc * 64, j, bar, stream_once);
-          tma_load_3d_pair_hint(a + 8192, &tmA, m0 + 64, kc * 64, j, bar, stream_once);
+          tma_load_3d_pair_hint(a, &tmA, m0, kc * 64, q.j, bar, stream_once);
+          tma_load_3d_pair_hint(a + 8192, &tmA, m0 + 64, kc * 64, q.j, bar, stream_once);
           for (int b = 0; b < nb0; ++b)
-            tma_load_3d_pair_hint(a + 16384 + b * 8192, &tmB, c0 + b * 64, kc * 64, j, bar, stream_once);
+            tma_load_3d_pair_hint(a + 16384 + b * 8192, &tmB, c0 + b * 64, kc * 64, q.j, bar, stream_once);
           for (int b = 0; b < nb1; ++b)
-            tma_load_3d_pair_hint(a + 16384 + (nb0 + b) * 8192, &tmB, c1 + b * 64, kc * 64, j, bar, stream_once);
+            tma_load_3d_pair_hint(a + 16384 + (nb0 + b) * 8192, &tmB, c1 + b * 64, kc * 64, q.j, bar, stream_once);
           if (++st == kWideStages) { st = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
-      int st = 0;
-      uint32_t ph = 0, aph = 0;
-      for (int u = pair_id; u < p.num_units && !failed; u += n_pairs) {
-        const int pass = (u % per_batch) / p.m_tiles;
-        int w0, w1;
-        wide_pass_widths(p.n_total, pass, &w0, &w1);
-        const int nb0 = (w0 / 2 + 63) / 64;
-        const uint32_t idesc0 = instr_desc_bf16(256, w0, 1, 1), idesc1 = instr_desc_bf16(256, w1 ? w1 : 32, 1, 1);
-        if (!mbar_wait(tempty, aph ^ 1u)) { failed = true; break; }
+      int st = 0, singles = 0;
+      uint32_t ph = 0, eph[2] = {0u, 0u};
+      for (int r = 0; r < rounds && !failed; ++r) {
+        const int u = wide_unit_of(r, pair_id, n_pairs);
+        if (u >= p.sch.num_units) continue;
+        const WideUnit q = wide_unit(p.batch, p.m_tiles, p.n_total, p.sch, u);
+        const bool both = q.w1 != 0;
+        const int a0 = both ? 0 : (singles++ & 1);  // a unit of one accumulator takes them in turn
+        const int nb0 = (q.w0 / 2 + 63) / 64;
+        const uint32_t idesc0 = instr_desc_bf16(256, q.w0, 1, 1), idesc1 = instr_desc_bf16(256, both ? q.w1 : 32, 1, 1);
+        const uint32_t acc0 = tmem_base + (uint32_t)a0 * 256u, acc1 = tmem_base + 256u;
+        if (!mbar_wait(tempty[a0], (a0 ? eph[1] : eph[0]) ^ 1u)) { failed = true; break; }
+        if (both && !mbar_wait(tempty[1], eph[1] ^ 1u)) { failed = true; break; }
         tc_fence_after();
         for (int kc = 0; kc < p.num_k; ++kc) {
           if (!mbar_wait(full[st], ph)) { failed = true; break; }
@@ -1416,52 +1382,107 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                          bd1 = smem_desc_sw128(a + 16384 + nb0 * 8192, 8192, 1024);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {  // 16 rows of K = 2048 bytes per instruction
-            mma_bf16_pair(tmem_base, ad + (uint64_t)(k4 * 128), bd0 + (uint64_t)(k4 * 128), idesc0, (kc | k4) != 0);
-            if (w1)
-              mma_bf16_pair(tmem_base + 256u, ad + (uint64_t)(k4 * 128), bd1 + (uint64_t)(k4 * 128), idesc1, (kc | k4) != 0);
+            mma_bf16_pair(acc0, ad + (uint64_t)(k4 * 128), bd0 + (uint64_t)(k4 * 128), idesc0, (kc | k4) != 0);
+            if (both)
+              mma_bf16_pair(acc1, ad + (uint64_t)(k4 * 128), bd1 + (uint64_t)(k4 * 128), idesc1, (kc | k4) != 0);
           }
           mma_commit_pair(empty[st], 3);
           if (++st == kWideStages) { st = 0; ph ^= 1u; }
         }
         if (failed) break;
-        mma_commit_pair(tfull, 3);
-        aph ^= 1u;
+        mma_commit_pair(tfull[a0], 3);
+        if (both) mma_commit_pair(tfull[1], 3);
+        if (a0 || both) eph[1] ^= 1u;
+        if (!a0) eph[0] ^= 1u;
       }
     }
   } else {
-    const int q = warp & 3, half = (warp - 2) >> 2;  // warps w and w + 4 share a quadrant and alternate 32-column chunks
+    const int q4 = warp & 3, half = (warp - 2) >> 2;  // warps w and w + 4 share a quadrant and alternate 32-column chunks
     if (p.side.slots) {
       const long long total = (long long)p.side.k * p.side.wstride, nthr = (long long)gridDim.x * (kWideThreads - 64);
       for (long long e = (long long)blockIdx.x * (kWideThreads - 64) + ((int)threadIdx.x - 64); e < total; e += nthr)
         head_reduce_one(p.side, (int)(e / p.side.wstride), (int)(e % p.side.wstride));
     }
-    uint32_t aph = 0;
-    for (int u = pair_id; u < p.num_units; u += n_pairs) {
-      const int j = p.batch - 1 - u / per_batch, mt = (u % per_batch) % p.m_tiles, pass = (u % per_batch) / p.m_tiles;
-      int w0, w1;
-      wide_pass_widths(p.n_total, pass, &w0, &w1);
-      if (!mbar_wait(tfull, aph)) { failed = true; break; }
-      tc_fence_after();
-      const int m = mt * 256 + (int)rank * 128 + q * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-      float *dst = p.out + (size_t)j * p.out_batch + m;
-      const int ch0 = w0 >> 5, chunks = ch0 + (w1 >> 5);
-      for (int ch = half; ch < chunks; ch += 2) {
-        const int col = ch < ch0 ? ch * 32 : 256 + (ch - ch0) * 32;  // accumulator column = column of the pass
-        const int n0 = pass * 512 + col;
-        if (n0 >= p.n_total) continue;  // (uniform per warp)
-        float v[32];
-        tmem_ld32(taddr + (uint32_t)col, v);
+    int singles = 0;
+    uint32_t fph[2] = {0u, 0u};
+    for (int r = 0; r < rounds && !failed; ++r) {
+      const int u = wide_unit_of(r, pair_id, n_pairs);
+      if (u >= p.sch.num_units) continue;
+      const WideUnit q = wide_unit(p.batch, p.m_tiles, p.n_total, p.sch, u);
+      const bool both = q.w1 != 0;
+      const int a0 = both ? 0 : (singles++ & 1);
+      const int m = q.mt * 256 + (int)rank * 128 + q4 * 32 + lane;
+      float *dst = p.out + (size_t)q.j * p.out_batch + m;
+      for (int x = 0; x < (both ? 2 : 1); ++x) {
+        const int acc = both ? x : a0, w = x ? q.w1 : q.w0, c = x ? q.c1 : q.c0;
+        if (!mbar_wait(tfull[acc], acc ? fph[1] : fph[0])) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)acc * 256u;
+        for (int ch = half; ch < (w >> 5); ch += 2) {
+          const int n0 = c + ch * 32;
+          if (n0 >= p.n_total) continue;  // (uniform per warp)
+          float v[32];
+          tmem_ld32(taddr + (uint32_t)(ch * 32), v);
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (n0 + i < p.n_total) dst[(size_t)(n0 + i) * p.out_ld] = v[i];
+          for (int i = 0; i < 32; ++i)
+            if (n0 + i < p.n_total) dst[(size_t)(n0 + i) * p.out_ld] = v[i];
+        }
+        tc_fence_before();
+        mbar_arrive_cluster(map_to_rank(tempty[acc], 0));
+        if (acc) fph[1] ^= 1u; else fph[0] ^= 1u;
       }
-      tc_fence_before();
-      mbar_arrive_cluster(map_to_rank(tempty, 0));
-      aph ^= 1u;
     }
   }
   pair_teardown(warp, tmem_base, failed, p.status);
+}
+
+// Which whole passes to cut in halves.  Cost of a unit per K chunk, in SM cycles: the slower of feeding shared
+// memory (measured: about 41 bytes per cycle and SM in these kernels) and the tensor cores (a 256 x w x 16
+// instruction takes w / 2 cycles), plus reading the accumulators out.  Candidates: keep all whole passes, or
+// cut the last t of them, t up to two rounds of pairs; each is dealt as the kernel deals and the one with
+// the shortest longest pair wins (ties: fewer cuts, i.e. less traffic).
+static double wide_unit_cost(int w0, int w1, int num_k) {
+  const int nb = (w0 / 2 + 63) / 64 + (w1 / 2 + 63) / 64;
+  const double fill = (16384.0 + 8192.0 * nb) / 41.0, mma = 2.0 * (w0 + w1);
+  return (fill > mma ? fill : mma) * num_k + 20.0 * (w0 + w1);
+}
+static WideSchedule wide_schedule(int batch, int m_tiles, int n_total, int num_k, int max_pairs) {
+  WideSchedule s;
+  s.full_passes = n_total / 512;
+  const int whole = batch * m_tiles * s.full_passes;
+  int rw0 = 0, rw1 = 0;
+  if (n_total % 512) wide_pass_widths(n_total, s.full_passes, &rw0, &rw1);
+  s.n_ragged = (n_total % 512) ? batch * m_tiles : 0;
+  const double c_whole = wide_unit_cost(256, 256, num_k), c_half = wide_unit_cost(256, 0, num_k),
+               c_ragged = s.n_ragged ? wide_unit_cost(rw0, rw1, num_k) : 0.0;
+  s.ragged_first = c_ragged >= c_half ? 1 : 0;
+  WideSchedule best = s;
+  double best_span = -1.0;
+  std::vector<double> load;
+  const int t_max = whole < 2 * max_pairs ? whole : 2 * max_pairs;
+  for (int t = 0; t <= t_max; ++t) {
+    s.n_whole = whole - t;
+    s.n_half = 2 * t;
+    s.num_units = s.n_whole + s.n_ragged + s.n_half;
+    s.pairs = s.num_units < max_pairs ? s.num_units : max_pairs;
+    if (s.pairs < 1) s.pairs = 1;
+    load.assign(s.pairs, 0.0);
+    const int second = s.ragged_first ? s.n_ragged : s.n_half;
+    for (int u = 0; u < s.num_units; ++u) {
+      const int r = u / s.pairs, pos = u % s.pairs, pair = (r & 1) ? s.pairs - 1 - pos : pos;
+      const double c = u < s.n_whole ? c_whole
+                       : (u < s.n_whole + second ? (s.ragged_first ? c_ragged : c_half)
+                                                 : (s.ragged_first ? c_half : c_ragged));
+      load[pair] += c;
+    }
+    double span = 0.0;
+    for (double v : load) span = v > span ? v : span;
+    if (best_span < 0.0 || span < best_span * (1.0 - 1e-9)) {
+      best_span = span;
+      best = s;
+    }
+  }
+  return best;
 }
 
 // The opt-in shared-memory size of a kernel is set once per device and kernel, not on every launch.
@@ -1581,9 +1602,10 @@ int head_grid(int k, int rows, int sms) {
 struct DenseState {
   struct {
     bool valid = false;
-    int k = 0, rows = 0, d = 0, C = 0;
+    int k = 0, rows = 0, d = 0, C = 0, sms = 0;
     const void *X = nullptr, *scratch = nullptr;
     CUtensorMap tmXa, tmXb, tmW, tmWh, tmR;
+    WideSchedule wide;  // units of the backward contraction (CTA-pair path)
   } sm;
   struct {
     bool valid = false;
@@ -1591,6 +1613,7 @@ struct DenseState {
     const void *Xb = nullptr, *scratch = nullptr;
     int max_slots = 0;
     CUtensorMap tmXa, tmXb, tmW, tmWh, tmH, tmHa, tmD1, tmD1s, tmD2, tmW2t, tmW2k;
+    WideSchedule wide;  // units of the [dW1; db1] contraction (CTA-pair path)
   } mlp;
   // bf16 copy [X 1] of an MLP's data matrix made by prepare_mlp_data (owned here)
   __nv_bfloat16 *Xb_prep = nullptr;
@@ -1598,6 +1621,28 @@ struct DenseState {
   const void *prep_src = nullptr;
   int prep_k = 0, prep_rows = 0, prep_d = 0;
 };
+
+// The unit list of the wide backward contraction as the kernel walks it, for inspection: row u of `units`
+// gets {pair, round, batch j, M block, c0, w0, c1, w1}.  Returns the number of units (rows written: at most cap).
+int wide_schedule_units(int batch, int m_tiles, int n_total, int num_k, int max_pairs, int *units, int cap,
+                        int *pairs_out) {
+  const WideSchedule s = wide_schedule(batch, m_tiles, n_total, num_k, max_pairs);
+  if (pairs_out) *pairs_out = s.pairs;
+  const int rounds = (s.num_units + s.pairs - 1) / s.pairs;
+  int n = 0;
+  for (int r = 0; r < rounds; ++r)
+    for (int pair = 0; pair < s.pairs; ++pair) {
+      const int u = wide_unit_of(r, pair, s.pairs);
+      if (u >= s.num_units) continue;
+      if (n < cap) {
+        const WideUnit q = wide_unit(batch, m_tiles, n_total, s, u);
+        int *row = units + (size_t)n * 8;
+        row[0] = pair; row[1] = r; row[2] = q.j; row[3] = q.mt; row[4] = q.c0; row[5] = q.w0; row[6] = q.c1; row[7] = q.w1;
+      }
+      ++n;
+    }
+  return n;
+}
 
 void dense_state_free(DenseState *st) {
   if (!st) return;
@@ -1633,7 +1678,8 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   *G_out = G;
 
   auto &c = st->sm;
-  if (!(c.valid && c.k == k && c.rows == rows && c.d == d && c.C == C && c.X == X && c.scratch == scratch)) {
+  if (!(c.valid && c.k == k && c.rows == rows && c.d == d && c.C == C && c.sms == sms && c.X == X &&
+        c.scratch == scratch)) {
     c.valid = false;
     const uint64_t xdims[3] = {(uint64_t)d, (uint64_t)rows, (uint64_t)k};
     const uint32_t xbox_a[3] = {64, 128, 1}, xbox_b[3] = {64, 64, 1};
@@ -1645,7 +1691,8 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
         !make_map(&c.tmW, Wt, 2, wdims, wbox) || !make_map(&c.tmWh, Wt, 2, wdims, wbox_h) ||
         !make_map(&c.tmR, R, 3, rdims, rbox))
       return cudaErrorInvalidValue;
-    c.k = k; c.rows = rows; c.d = d; c.C = C; c.X = X; c.scratch = scratch;
+    if (C == 256 && sms >= 2) c.wide = wide_schedule(k, 1, d, (rows + 63) / 64, sms / 2);
+    c.k = k; c.rows = rows; c.d = d; c.C = C; c.sms = sms; c.X = X; c.scratch = scratch;
     c.valid = true;
   }
 
@@ -1672,6 +1719,15 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   }
   if (e != cudaSuccess) return e;
 
+  if (pair) {
+    // G_j^T = R_j^T X_j: the residual (C = 256 classes) on the M side, the data matrix on the N side in passes of
+    // 512 features; the transposed store puts element (class, feature) at G[feature][class]
+    TnWideParams wp;
+    wp.batch = k; wp.m_tiles = 1; wp.sch = c.wide; wp.num_k = (rows + 63) / 64;
+    wp.n_total = d; wp.out = G; wp.out_batch = (size_t)d * C; wp.out_ld = C; wp.status = status;
+    wp.side = HeadSlots{};
+    return launch_pair(tn_wide_pair_kernel, kWideThreads, wp.sch.num_units, sms, c.tmR, c.tmXb, wp, stream, kSmemWide);
+  }
   TnParams t;
   t.batch = k; t.n_tiles = 1;
   t.num_k = (rows + 63) / 64;
@@ -1679,10 +1735,6 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
   t.m_store = d; t.n_store = C;
   t.out = G; t.out_batch = (size_t)d * C; t.out_ld = C;
   t.status = status;
-  if (pair) {
-    t.m_tiles = (d + 255) / 256; t.num_tiles = k * t.m_tiles;
-    return launch_pair(tn_gemm_pair_kernel, kTcThreads, t.num_tiles, sms, c.tmXb, c.tmR, t, stream);
-  }
   if ((e = ensure_smem_attr(tn_gemm_kernel, kSmemTc)) != cudaSuccess) return e;
   t.m_tiles = (d + 127) / 128; t.num_tiles = k * t.m_tiles;
   launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, c.tmXb, c.tmR, t);
@@ -1807,6 +1859,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
       if (!make_map(&c.tmW2t, W2t, 2, w2tdims, box_w2t) || !make_map(&c.tmW2k, W2k, 2, w2kdims, box_w2k))
         return cudaErrorInvalidValue;
     }
+    if (hidden % 256 == 0 && sms >= 2) c.wide = wide_schedule(k, hidden / 256, d + 1, (rows + 63) / 64, sms / 2);
     c.k = k; c.rows = rows; c.d = d; c.hidden = hidden; c.C = C; c.sms = sms; c.Xb = Xb; c.scratch = scratch;
     c.valid = true;
   }
@@ -1892,11 +1945,10 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   if (pair) {
     // delta1 on the M side (hidden is a multiple of 256), [X 1] on the N side in passes of 512 columns
     TnWideParams wp;
-    wp.batch = k; wp.m_tiles = hidden / 256; wp.n_passes = (d + 1 + 511) / 512;
-    wp.num_units = k * wp.m_tiles * wp.n_passes; wp.num_k = (rows + 63) / 64;
+    wp.batch = k; wp.m_tiles = hidden / 256; wp.sch = c.wide; wp.num_k = (rows + 63) / 64;
     wp.n_total = d + 1; wp.out = G; wp.out_batch = lpad; wp.out_ld = hidden; wp.status = status;
     wp.side = head_slots;
-    e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.num_units, sms, c.tmD1, c.tmXb, wp, stream, kSmemWide);
+    e = launch_pair(tn_wide_pair_kernel, kWideThreads, wp.sch.num_units, sms, c.tmD1, c.tmXb, wp, stream, kSmemWide);
   } else {
     if ((e = ensure_smem_attr(tn_gemm_kernel, kSmemTc)) != cudaSuccess) return e;
     launch_k(tn_gemm_kernel, t.num_tiles < sms ? t.num_tiles : sms, kTcThreads, kSmemTc, stream, c.tmXb, c.tmD1, t);

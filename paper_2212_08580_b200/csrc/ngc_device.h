@@ -95,6 +95,11 @@ cudaError_t launch_softmax_grad(int k, int rows, int d, int C, const void *X, co
                                 unsigned char *scratch, float **G_out, int *status, int sms, cudaStream_t stream,
                                 DenseState **state);
 
+// Host only: how the wide backward contraction (D^T = A^T B, M blocks of 256, N passes of 512 columns, some cut in
+// halves) splits a problem into units and deals them to `max_pairs` CTA pairs; see ngc_dense_schedule in ngc.h.
+int wide_schedule_units(int batch, int m_tiles, int n_total, int num_k, int max_pairs, int *units, int cap,
+                        int *pairs_out);
+
 // Monte Carlo of the stopping rule (Section IV): latency (gamma + eps + decode instant, +inf if never) and
 // chosen level (-1 if none) of `trials` seeded straggler patterns, into device buffers.
 cudaError_t launch_latency_mc(const ngc_plan_s &plan, uint64_t seed, long long trials, double shift, double rate,

@@ -28,6 +28,8 @@ CASES = [
     (4, [1], 520, 1032, 256, 1),       # CTA-pair kernels: ragged 256-row blocks, five feature blocks (the last 8 wide)
     (2, [1], 200, 128, 256, 2),        # k = 2 n with full-width classes, less than one 256-row block
     (2, [0], 256, 64, 256, 2),         # ... exactly one block, a single K chunk in the forward pass
+    (90, [1], 192, 1032, 256, 1),      # backward units on the CTA pairs in four and five rounds: whole passes, halves
+                                       # and ragged passes after one another, the one-accumulator units taking turns
 ]
 
 
