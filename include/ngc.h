@@ -215,8 +215,13 @@ int ngc_step_host(ngc_plan_t *plan, const ngc_model_t *model, const float *theta
  *      cancel, so they are added across ranks before anything is rounded to fp32;
  *   4. (caller) one all-reduce (sum) of partial_dev over the ranks gives the decoded gradient.
  * Results equal those of ngc_grad_encode + ngc_decode on one GPU up to summation order.  n_local + s_l <=
- * NGC_MAX_N.  Asynchronous on the stream except for a short synchronisation in step 3.
+ * NGC_MAX_N.  Asynchronous on the stream, except that the first step-3 call for a (level, first_worker, n_local)
+ * uploads that shard's rows of the code matrix after waiting for the stream (a rank asks for the same shard in
+ * every iteration, so this happens once per level; such a call cannot be captured into a graph).
+ * ngc_shard_prepare_data is ngc_prepare_data for a shard: X_local_dev holds the rank's n_local * q partitions.
  */
+int ngc_shard_prepare_data(ngc_plan_t *plan, const ngc_model_t *model, const void *X_local_dev, int n_local,
+                           void *cuda_stream);
 int ngc_shard_gradients(ngc_plan_t *plan, const ngc_model_t *model, const void *theta_dev, const void *X_local_dev,
                         const void *y_local_dev, int n_local, float *G_dev, int64_t ld, void *cuda_stream);
 int ngc_shard_encode_decode(ngc_plan_t *plan, const ngc_model_t *model, int layer, int first_worker, int n_local,

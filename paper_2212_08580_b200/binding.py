@@ -69,6 +69,7 @@ def load_library() -> C.CDLL:
         "ngc_coded_dtype": (i32, [vp, P(Model)]),
         "ngc_select": (i32, [vp, P(dbl), P(StepInfo)]),
         "ngc_prepare_data": (i32, [vp, P(Model), vp, vp]),
+        "ngc_shard_prepare_data": (i32, [vp, P(Model), vp, i32, vp]),
         "ngc_shard_gradients": (i32, [vp, P(Model), vp, vp, vp, i32, vp, i64, vp]),
         "ngc_shard_encode_decode": (i32, [vp, P(Model), i32, i32, i32, vp, i64, P(C.c_int32), i32, vp, vp, vp]),
         "ngc_grad_encode": (i32, [vp, P(Model), vp, vp, vp, i32, vp, vp]),
@@ -234,6 +235,12 @@ class Plan:
         """ngc_prepare_data: what the library derives from the data matrix alone, made once (X=None drops it)."""
         self._check(self._lib.ngc_prepare_data(self._h, C.byref(model), _addr(X) if X is not None else None, stream),
                     "ngc_prepare_data")
+
+    def shard_prepare_data(self, model: Model, X_local, n_local: int, stream: int = 0):
+        """ngc_shard_prepare_data: prepare_data for a shard of n_local partition groups."""
+        self._check(self._lib.ngc_shard_prepare_data(self._h, C.byref(model),
+                                                     _addr(X_local) if X_local is not None else None, n_local, stream),
+                    "ngc_shard_prepare_data")
 
     def shard_gradients(self, model: Model, theta, X_local, y_local, n_local: int, G, ld: int, stream: int = 0):
         self._check(self._lib.ngc_shard_gradients(self._h, C.byref(model), _addr(theta), _addr(X_local), _addr(y_local),

@@ -349,25 +349,37 @@ int ngc_shard_encode_decode(ngc_plan_t *p, const ngc_model_t *m, int layer, int 
   if ((rc = pack_set(p, layer, S, nS, mask.w)) != NGC_OK) return rc;
   if ((rc = ensure_tables(p)) != NGC_OK) return rc;
   if ((rc = ensure_batch(p, 1)) != NGC_OK) return rc;
+  const size_t table = (size_t)NGC_MAX_N * (NGC_MAX_S + 1);
   if (!p->d_shard_coef) {
-    NGC_CUDA(p, cudaMalloc(&p->d_shard_coef, (size_t)NGC_MAX_N * (NGC_MAX_S + 1) * sizeof(double)));
+    NGC_CUDA(p, cudaMalloc(&p->d_shard_coef, (size_t)p->L * table * sizeof(double)));
     NGC_CUDA(p, cudaMalloc(&p->d_shard_a, (size_t)NGC_MAX_N * sizeof(double)));
+    p->shard_key.assign((size_t)2 * p->L, -1);
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  // Rows first_worker .. first_worker + n_local - 1 of B (window form), then s all-zero rows: the encode kernels
-  // index the partial gradients cyclically over `rows` entries, and only the zero rows ever wrap.
-  p->shard_coef_host.assign((size_t)rows * (s + 1), 0.0);
-  for (int r = 0; r < n_local; ++r) {
-    const int i = (first_worker + r) % n;
-    for (int t = 0; t <= s; ++t) p->shard_coef_host[(size_t)r * (s + 1) + t] = lv.coef[(size_t)i * (s + 1) + t];
+  double *d_coef = p->d_shard_coef + (size_t)layer * table;
+  if (p->shard_key[2 * layer] != first_worker || p->shard_key[2 * layer + 1] != n_local) {
+    // Rows first_worker .. first_worker + n_local - 1 of B (window form), then s all-zero rows: the encode kernels
+    // index the partial gradients cyclically over `rows` entries, and only the zero rows ever wrap.  A rank asks
+    // for the same shard in every iteration, so each level's table is uploaded once; when the shard does change,
+    // work queued on the stream may still read the old table: wait for it first.
+    p->shard_coef_host.assign((size_t)rows * (s + 1), 0.0);
+    for (int r = 0; r < n_local; ++r) {
+      const int i = (first_worker + r) % n;
+      for (int t = 0; t <= s; ++t) p->shard_coef_host[(size_t)r * (s + 1) + t] = lv.coef[(size_t)i * (s + 1) + t];
+    }
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    NGC_CUDA(p, cudaStreamIsCapturing(stream, &cap));
+    if (cap != cudaStreamCaptureStatusNone) return NGC_ERR_INVALID;  // serve the shard once eagerly before capturing
+    NGC_CUDA(p, cudaStreamSynchronize(stream));
+    NGC_CUDA(p, cudaMemcpy(d_coef, p->shard_coef_host.data(), p->shard_coef_host.size() * sizeof(double),
+                           cudaMemcpyHostToDevice));
+    p->shard_key[2 * layer] = first_worker;
+    p->shard_key[2 * layer + 1] = n_local;
   }
-  NGC_CUDA(p, cudaMemcpyAsync(p->d_shard_coef, p->shard_coef_host.data(), p->shard_coef_host.size() * sizeof(double),
-                              cudaMemcpyHostToDevice, stream));
-  NGC_CUDA(p, cudaStreamSynchronize(stream));  // the host vector is reused by the next call
   const int cdt = ngc_coded_dtype(p, m);
   ngc::RowSplit split;
   split.T = rows; split.rows_g = 1; split.grid = rows; split.P = 1;
-  NGC_CUDA(p, ngc::launch_encode_long(split, G_window, ld, p->d_shard_coef, rows, s, l, coded, cdt, stream));
+  NGC_CUDA(p, ngc::launch_encode_long(split, G_window, ld, d_coef, rows, s, l, coded, cdt, stream));
   // the decoding vector of the whole responsive set; this shard applies the weights of its own workers
   NGC_CUDA(p, ngc::launch_decode_solve(*p, layer, nullptr, mask, 1, p->d_a, p->d_resid, p->d_maxres, stream));
   NGC_CUDA(p, cudaMemsetAsync(p->d_shard_a, 0, (size_t)NGC_MAX_N * sizeof(double), stream));
@@ -394,6 +406,19 @@ int ngc_prepare_data(ngc_plan_t *p, const ngc_model_t *m, const void *X, void *c
   NGC_CUDA(p, ngc::prepare_mlp_data(reinterpret_cast<ngc::DenseState **>(&p->dense_state), p->k, m->rows_per_partition,
                                     m->d, static_cast<const float *>(X), static_cast<cudaStream_t>(cuda_stream)));
   if (X) p->launches += 1;
+  return NGC_OK;
+}
+
+int ngc_shard_prepare_data(ngc_plan_t *p, const ngc_model_t *m, const void *X_local, int n_local, void *cuda_stream) {
+  if (!p || n_local < 1 || n_local > p->n) return NGC_ERR_INVALID;
+  int rc = check_model(p, m);
+  if (rc != NGC_OK) return rc;
+  if (m->kind != NGC_MLP) return NGC_OK;
+  if (m->x_dtype != NGC_F32 || m->d % 8 != 0 || (X_local && !aligned16(X_local))) return NGC_ERR_INVALID;
+  NGC_CUDA(p, ngc::prepare_mlp_data(reinterpret_cast<ngc::DenseState **>(&p->dense_state), n_local * (p->k / p->n),
+                                    m->rows_per_partition, m->d, static_cast<const float *>(X_local),
+                                    static_cast<cudaStream_t>(cuda_stream)));
+  if (X_local) p->launches += 1;
   return NGC_OK;
 }
 

@@ -37,8 +37,9 @@ struct ngc_plan_s {
   int *d_status = nullptr;     // [0] timeout flag, [1] scratch
   double *d_maxres = nullptr;  // largest residual seen by asynchronous decodes
   // sharded operation: coefficient rows and decoding weights of the workers one shard holds
-  double *d_shard_coef = nullptr;  // NGC_MAX_N x (NGC_MAX_S + 1)
+  double *d_shard_coef = nullptr;  // per level: NGC_MAX_N x (NGC_MAX_S + 1), the rows of B of the shard last served
   double *d_shard_a = nullptr;     // NGC_MAX_N
+  std::vector<int> shard_key;      // per level: {first_worker, n_local} of the table on the device, -1 = none
   std::vector<double> shard_coef_host;
   void *dense_state = nullptr; // ngc::DenseState*: cached tensor maps of the dense launchers, data prepared once
   void *d_gpart = nullptr;     // per-chunk partial decodes of the fused encode + decode (dense models)

@@ -112,6 +112,8 @@ class ShardedStep:
         self.coded = torch.empty((self.n_local + s_max, self.l), dtype=cdt, device=device)
         self.partial = torch.empty(self.l, dtype=cdt, device=device)
         self.grad = torch.empty(self.l, dtype=torch.float32, device=device)
+        # the rank's data does not change between iterations (Section II-C): derive what depends on it alone once
+        self.plan.shard_prepare_data(self.m, self.X, self.n_local, torch.cuda.current_stream().cuda_stream)
 
     def step(self, theta, task_times, group=None):
         """Returns the stopping rule's result; self.grad holds the decoded gradient on every rank."""

@@ -93,3 +93,34 @@ def test_single_rank_sharded_step_is_the_whole_problem():
         torch.cuda.synchronize()
         assert info.sigma == (1 if len(stragglers) < 2 else 2)
         assert rel_l2(st.grad.cpu().numpy(), G.sum(axis=0)) < 1e-5
+
+
+def test_one_plan_serving_different_shards_in_turn_reloads_its_code_rows():
+    """The rows of B a shard needs stay on the device per level; a plan asked for another shard must replace them."""
+    w = _case("logistic", "f32", 9, [2], 96, 256, 11)
+    X, y, theta = ngc_inputs.make_data(w, "cuda")
+    m = model_of(w)
+    l = w.n_params
+    lay = ShardLayout(w.n, 2)
+    G = oracle_G(w, X, y, theta)
+    p = ngc.Plan(w.n, w.levels, seed=w.seed)
+    cdt = coded_torch_dtype(p.coded_dtype(m))
+    ld = (l + 3) // 4 * 4
+    t = ngc_inputs.set_times(w.n, 3, [1, 7])
+    info = p.select(t)
+    S, s = info.responsive(), info.sigma
+    Gd = torch.zeros((w.n, ld), dtype=torch.float32, device="cuda")
+    p.shard_gradients(m, theta, X, y, w.n, Gd, ld)                      # all groups at once: the rows to hand out
+    for _ in range(2):                                                  # shard 0, shard 1, shard 0, shard 1
+        total = torch.zeros(l, dtype=torch.float64, device="cuda")
+        for r in range(2):
+            first, cnt = lay.first(r), lay.count(r)
+            win = torch.zeros((cnt + s, ld), dtype=torch.float32, device="cuda")
+            rows = [(first + i) % w.n for i in range(cnt + s)]
+            win.copy_(Gd[rows])
+            coded = torch.empty((cnt + s, l), dtype=cdt, device="cuda")
+            part = torch.empty(l, dtype=cdt, device="cuda")
+            p.shard_encode_decode(m, info.layer, first, cnt, win, ld, S, coded, part)
+            torch.cuda.synchronize()
+            total += part.double()
+        assert rel_l2(total.cpu().numpy(), G.sum(axis=0)) < 1e-5
