@@ -476,8 +476,8 @@ def measure_side_workload(name, dev, peaks, which, smi_index, args):
     sampler.start()
     time.sleep(0.05)
     total_ms, levels = timed_steps(pb, pats, steps)
+    kern_ms, kern_n = kernel_bracket(pb, pats, min(steps, 50))   # right behind the timed steps: the same clock state
     med = per_step_median_ms(pb, pats, steps)
-    kern_ms, kern_n = kernel_bracket(pb, pats, min(steps, 50))
     clocks = sampler.stop()
     host_us = host_queue_us(pb, pats, steps)
     per_level = grad_encode_per_level(pb, peaks)
@@ -546,9 +546,10 @@ def run_cuda(args):
         dist.barrier()
     ms_total = rank_max(ms_local, world, dev)
     launches = pb.plan.launch_count() - launches0
-    # ---- separate passes: per-step median, then the event brackets around the gradient kernels
-    median_ms = per_step_median_ms(pb, pats[args.warmup:], args.median_steps) if args.median_steps else None
+    # ---- separate passes: the event brackets around the gradient kernels (right behind the timed steps, so that
+    # they see the clock state the timed steps saw), then the per-step median
     kern_ms, kern_n = kernel_bracket(pb, pats[args.warmup:], min(max(args.steps, 20), 100))
+    median_ms = per_step_median_ms(pb, pats[args.warmup:], args.median_steps) if args.median_steps else None
     clocks = sampler.stop() if rank == 0 else {}
     host_us = host_queue_us(pb, pats[args.warmup:], min(max(args.steps, 20), 200))
     peaks, which = measured_peaks()
