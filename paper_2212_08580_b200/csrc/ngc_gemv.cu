@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
   unsigned char *tail = smem + (size_t)p.stages * p.stage_bytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(tail);        // kMaxStages
   float *red = reinterpret_cast<float *>(tail + 128);         // [R][kWarps] per-warp partial dot products
-  float *resv = red + R * kWarps;                             // [R] residuals of the tile's rows
+  float *resv = red + 2 * R * kWarps;                         // [R] residuals of the tile's rows (behind two red buffers)
   volatile int *abort_flag = reinterpret_cast<volatile int *>(resv + R);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -232,7 +232,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
     cons.next(R, row0, nrows, seg_last, g);
     // the warps that will finish the row sums fetch the labels early
     float yrow = 0.f;
-    if (warp < R && lane == 0 && warp < nrows) yrow = __ldg(p.y + row0 + warp);
+    if (R == 2) {
+      if ((lane >> 4) < nrows) yrow = __ldg(p.y + row0 + (lane >> 4));
+    } else if (warp < R && lane == 0 && warp < nrows) {
+      yrow = __ldg(p.y + row0 + warp);
+    }
 
     if (!mbar_wait(smem_u32(&bars[st]), parity)) {
       failed = true;
@@ -260,21 +264,41 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
       pd[r] = lo + hi;
     }
     const float rowsum = warp_reduce_rows<R>(pd, lane);
-    if ((lane & (31 >> Log2<R>::v)) == 0) red[(lane >> (5 - Log2<R>::v)) * kWarps + warp] = rowsum;
-    __syncthreads();
-    if (warp < R) {  // warp r finishes row r: sum over the kWarps partials, then the residual
-      float z = (lane < kWarps) ? red[warp * kWarps + lane] : 0.f;
+    float res_r[R];
+    if (R == 2) {
+      // Two rows per tile: one barrier.  Every warp adds up the 16 per-warp parts of both rows itself (lanes 0-15
+      // row 0, lanes 16-31 row 1) from a buffer that alternates with the tile's parity, so nobody waits for two
+      // finishing warps and a second barrier.
+      float *rb = red + (t & 1) * (R * kWarps);
+      if ((lane & 15) == 0) rb[(lane >> 4) * kWarps + warp] = rowsum;
+      __syncthreads();
+      if (*abort_flag) break;
+      float z = rb[lane];  // kWarps == 16: element (lane >> 4) * kWarps + (lane & 15)
 #pragma unroll
-      for (int off = kWarps / 2; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
-      if (lane == 0) {
-        // (one code path for both activations: as two template instances the least-squares one, although the
-        // simpler, was compiled with spills at the 128-register cap of the widest bf16 shape)
-        const float res = (p.act ? 1.f / (1.f + expf(-z)) : z) - yrow;
-        resv[warp] = (warp < nrows) ? res : 0.f;
+      for (int off = 8; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+      float res = (p.act ? 1.f / (1.f + expf(-z)) : z) - yrow;
+      if ((lane >> 4) >= nrows) res = 0.f;
+      res_r[0] = __shfl_sync(0xffffffffu, res, 0);
+      res_r[R - 1] = __shfl_sync(0xffffffffu, res, 16);
+    } else {
+      if ((lane & (31 >> Log2<R>::v)) == 0) red[(lane >> (5 - Log2<R>::v)) * kWarps + warp] = rowsum;
+      __syncthreads();
+      if (warp < R) {  // warp r finishes row r: sum over the kWarps partials, then the residual
+        float z = (lane < kWarps) ? red[warp * kWarps + lane] : 0.f;
+#pragma unroll
+        for (int off = kWarps / 2; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+        if (lane == 0) {
+          // (one code path for both activations: as two template instances the least-squares one, although the
+          // simpler, was compiled with spills at the 128-register cap of the widest bf16 shape)
+          const float res = (p.act ? 1.f / (1.f + expf(-z)) : z) - yrow;
+          resv[warp] = (warp < nrows) ? res : 0.f;
+        }
       }
+      __syncthreads();
+      if (*abort_flag) break;
+#pragma unroll
+      for (int r = 0; r < R; ++r) res_r[r] = resv[r];
     }
-    __syncthreads();
-    if (*abort_flag) break;
     if (sizeof(XT) == 2) {
       // keep the packed words, not their unpacked copies, live across the barriers
 #pragma unroll
@@ -285,7 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_pair_kernel(const GemvParams
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      const float res = resv[r];
+      const float res = res_r[r];
       const f32x2 res2 = pack2(res, res);
 #pragma unroll
       for (int c = 0; c < VPT; ++c) {

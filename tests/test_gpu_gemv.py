@@ -31,6 +31,8 @@ CASES = [
     ("logistic", "f32", 3, [1], 1, 4, 1),                # one row, one vector
     ("lsq", "f32", 128, [1, 32], 3, 64, 1),              # the largest n and the largest tolerance the library takes
     ("lsq", "bf16", 2, [0, 1], 5000, 16384, 1),          # many rows per CTA range, widest rows
+    ("logistic", "bf16", 6, [1, 2], 75, 16384, 1),       # two-row tiles (one barrier per tile) with the sigmoid, odd row count
+    ("logistic", "f32", 5, [1], 33, 8192, 1),            # the same path on fp32 rows
 ]
 
 
