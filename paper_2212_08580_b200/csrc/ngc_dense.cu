@@ -341,7 +341,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {  // all 32 lanes walk the loop (uniform operands); one elected lane issues the tensor-core instructions
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
@@ -702,7 +702,7 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {  // all 32 lanes walk the loop (uniform operands); one elected lane issues the tensor-core instructions
       const uint32_t idesc_z = instr_desc_bf16(128, 16, 0, 0), idesc_w = instr_desc_bf16(128, 16, 1, 1);
       const int nmb = p.hidden / 128;
       uint32_t ph = 0, dph = 0;
@@ -974,7 +974,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {  // all 32 lanes walk the loop (uniform operands); one elected lane issues the tensor-core instructions
       const uint32_t idesc = instr_desc_bf16(128, p.N, 1, 1);
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
@@ -1137,7 +1137,7 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {  // all 32 lanes walk the loop (uniform operands); one elected lane issues
       const uint32_t idesc = instr_desc_bf16(256, 256, 0, 0);
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
@@ -1358,7 +1358,7 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {  // all 32 lanes walk the loop (uniform operands); one elected lane issues
       int st = 0, singles = 0;
       uint32_t ph = 0, eph[2] = {0u, 0u};
       for (int r = 0; r < rounds && !failed; ++r) {
