@@ -42,7 +42,7 @@ FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
 # dram__bytes_read.sum + dram__bytes_write.sum per full-size launch of the timed kernel (dense workloads: summed
 # over the gradient kernels the events bracket), from the ncu captures summarised under profiles/; None = the
 # kernels have changed since the counters were taken.
-TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000, "softmax50": 998_000_000, "mlp30": 359_500_000}
+TRAFFIC_BYTES = {"logistic20": 2_689_000_000, "lsq100": 6_585_000_000, "softmax50": 997_200_000, "mlp30": 357_700_000}
 
 
 # ----------------------------------------------------------------------------- small helpers
