@@ -347,11 +347,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
         const int nt = tile % p.n_tiles;
         const uint32_t idesc = instr_desc_bf16(128, min(256, p.n_total - nt * 256), 0, 0);
-        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
+        if (!mbar_wait_warp(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
         tc_fence_after();
         const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
         for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
+          if (!mbar_wait_warp(s.full[st], ph)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
           const uint64_t ad = smem_desc_sw128(a, 16, 1024), bd = smem_desc_sw128(a + kABytes, 16, 1024);
@@ -706,10 +706,10 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       const uint32_t idesc_z = instr_desc_bf16(128, 16, 0, 0), idesc_w = instr_desc_bf16(128, 16, 1, 1);
       const int nmb = p.hidden / 128;
       uint32_t ph = 0, dph = 0;
-      if (!mbar_wait(w_full, 0)) failed = true;
+      if (!mbar_wait_warp(w_full, 0)) failed = true;
       for (int tile = t_begin; tile < t_end && !failed; ++tile) {
         for (int g = 0; g < ngroups && !failed; ++g) {
-          if (!mbar_wait(h_full[g], ph)) { failed = true; break; }
+          if (!mbar_wait_warp(h_full[g], ph)) { failed = true; break; }
           tc_fence_after();
           for (int kc = g * 2; kc < min(nchunk, g * 2 + 2); ++kc) {
             const uint64_t ad = smem_desc_sw128(smem_u32(htile + kc * 16384), 16, 1024);
@@ -721,13 +721,13 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
         }
         if (failed) break;
         mma_commit(z_full);
-        if (!mbar_wait(d2_full, ph)) { failed = true; break; }
+        if (!mbar_wait_warp(d2_full, ph)) { failed = true; break; }
         tc_fence_after();
         const bool first = tile == t_begin || tile % tpp == 0;  // first tile of its partition in this CTA
         const uint64_t ad1 = smem_desc_sw128(smem_u32(d2tile), 16, 1024);      // delta2, K-major (K = classes)
         const uint64_t bdw = smem_desc_sw128(smem_u32(d2tile), 16384, 1024);   // delta2, N-major (K = samples)
         for (int hh = 0; hh < nhalf; ++hh) {
-          if (!mbar_wait(d_empty, dph ^ 1u)) { failed = true; break; }
+          if (!mbar_wait_warp(d_empty, dph ^ 1u)) { failed = true; break; }
           tc_fence_after();
           const int nh = min(256, p.hidden - hh * 256);
           const uint64_t bd = smem_desc_sw128(smem_u32(w2k + hh * 32768), 16, 1024);
@@ -979,11 +979,11 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles && !failed; tile += gridDim.x) {
-        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
+        if (!mbar_wait_warp(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
         tc_fence_after();
         const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
         for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
+          if (!mbar_wait_warp(s.full[st], ph)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a = smem_u32(s.tiles + st * kStageBytes);
           // M/N-major: 64-element boxes 8192 B apart, 8-row K groups 1024 B apart
@@ -1142,11 +1142,11 @@ fwd_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int st = 0, buf = 0;
       uint32_t ph = 0, aph = 0;
       for (int tile = pair_id; tile < p.num_tiles && !failed; tile += n_pairs) {
-        if (!mbar_wait(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
+        if (!mbar_wait_warp(s.tempty[buf], aph ^ 1u)) { failed = true; break; }
         tc_fence_after();
         const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
         for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(s.full[st], ph)) { failed = true; break; }
+          if (!mbar_wait_warp(s.full[st], ph)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a = smem_u32(s.tiles + st * kPairStageBytes);
           const uint64_t ad = smem_desc_sw128(a, 16, 1024), bd = smem_desc_sw128(a + 16384, 16, 1024);
@@ -1370,11 +1370,11 @@ tn_wide_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int nb0 = (q.w0 / 2 + 63) / 64;
         const uint32_t idesc0 = instr_desc_bf16(256, q.w0, 1, 1), idesc1 = instr_desc_bf16(256, both ? q.w1 : 32, 1, 1);
         const uint32_t acc0 = tmem_base + (uint32_t)a0 * 256u, acc1 = tmem_base + 256u;
-        if (!mbar_wait(tempty[a0], (a0 ? eph[1] : eph[0]) ^ 1u)) { failed = true; break; }
-        if (both && !mbar_wait(tempty[1], eph[1] ^ 1u)) { failed = true; break; }
+        if (!mbar_wait_warp(tempty[a0], (a0 ? eph[1] : eph[0]) ^ 1u)) { failed = true; break; }
+        if (both && !mbar_wait_warp(tempty[1], eph[1] ^ 1u)) { failed = true; break; }
         tc_fence_after();
         for (int kc = 0; kc < p.num_k; ++kc) {
-          if (!mbar_wait(full[st], ph)) { failed = true; break; }
+          if (!mbar_wait_warp(full[st], ph)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a = smem_u32(tiles + st * kWideStageBytes);
           // M/N-major: 64-element boxes 8192 B apart, 8-row K groups 1024 B apart

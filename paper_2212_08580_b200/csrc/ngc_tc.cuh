@@ -52,6 +52,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long lo
   }
 }
 
+// The same for a warp that walks its loop with all lanes and meets at `elect.sync` afterwards: the decision is
+// the warp's (if one lane gave up, all do), so no lane is left waiting for the others at the next warp-wide instruction.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity));
+}
+
 // ---- L2 eviction priority ---------------------------------------------------------------------
 // A policy word for loads of data that is streamed once per kernel (the data matrix, an intermediate read
 // for the last time): such lines are the first to be evicted, so that they do not push out what the next
