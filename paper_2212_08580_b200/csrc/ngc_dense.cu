@@ -623,30 +623,31 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char *sm = smem_raw + ((1024u - (base & 1023u)) & 1023u);
-  const int nchunk = p.hidden / 64, nhalf = (p.hidden + 255) / 256, ngroups = (nchunk + 1) / 2;
+  const int nchunk = p.hidden / 64, nhalf = (p.hidden + 255) / 256, ngroups = nchunk;
   unsigned char *htile = sm;                                  // nchunk x [128 x 64] bf16
   unsigned char *d2tile = htile + (size_t)nchunk * 16384;     // [128 x 64] bf16 (16 columns used)
   unsigned char *w2k = d2tile + 16384;                        // nhalf x [256 x 64] bf16
   unsigned char *w2t = w2k + (size_t)nhalf * 32768;           // nchunk x [16 x 64] bf16
   uint64_t *bars = reinterpret_cast<uint64_t *>(w2t + (size_t)nchunk * 2048);
-  // The tile lives in shared memory as groups of two 64-column chunks.  Group g is loaded (h), consumed,
-  // overwritten in place (delta1), stored and reloaded with the next tile's h on its own barriers, so the
-  // memory traffic of the finished groups hides behind the arithmetic on the others.
-  const BarArray h_full{smem_u32(&bars[0])}, m_done{smem_u32(&bars[4])}, w_done{smem_u32(&bars[8])};
-  const uint32_t z_full = smem_u32(&bars[12]), d2_full = smem_u32(&bars[13]), d_full = smem_u32(&bars[14]),
-                 d_empty = smem_u32(&bars[15]), w_full = smem_u32(&bars[16]);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[17]);
-  float *b2s = reinterpret_cast<float *>(&bars[18]);          // 16 floats
-  float *dbx = reinterpret_cast<float *>(&bars[26]);          // [4 quadrants][16]: bias-gradient partial sums
-  const uint32_t epi_bar = smem_u32(&bars[58]);               // meeting point of the epilogue threads (bounded, unlike bar.sync)
+  // The tile lives in shared memory as 64-column chunks.  Chunk g is loaded (h), consumed, overwritten in place
+  // (delta1), stored and reloaded with the next tile's h on its own barriers, so the memory traffic of the
+  // finished chunks hides behind the arithmetic on the others, and what is left when the last chunk is done is
+  // one chunk's store and reload (with pairs of chunks it was two chunks' worth: a quarter of the tile's time).
+  const BarArray h_full{smem_u32(&bars[0])}, m_done{smem_u32(&bars[8])}, w_done{smem_u32(&bars[16])};
+  const uint32_t z_full = smem_u32(&bars[20]), d2_full = smem_u32(&bars[21]), d_full = smem_u32(&bars[22]),
+                 d_empty = smem_u32(&bars[23]), w_full = smem_u32(&bars[24]);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(&bars[25]);
+  float *b2s = reinterpret_cast<float *>(&bars[26]);          // 16 floats
+  float *dbx = reinterpret_cast<float *>(&bars[34]);          // [4 quadrants][16]: bias-gradient partial sums
+  const uint32_t epi_bar = smem_u32(&bars[66]);               // meeting point of the epilogue threads (bounded, unlike bar.sync)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
+    for (int g = 0; g < 8; ++g) {
       mbar_init(h_full[g], 1);
       mbar_init(m_done[g], kHeadEpiThreads);
-      mbar_init(w_done[g], 1);
+      if (g < 4) mbar_init(w_done[g], 1);
     }
     mbar_init(z_full, 1);
     mbar_init(d2_full, 128);
@@ -669,8 +670,8 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
             t_end = head_tile_begin((int)blockIdx.x + 1, p.num_tiles, grid);
 
   if (warp == 0 || warp == 2) {
-    // Two producers: warp 0 owns the even chunk groups, warp 2 the odd ones, so that one of them can wait for
-    // a store to release its group while the other already handles the next group.
+    // Two producers: warp 0 owns the even chunks, warp 2 the odd ones, so that one of them can wait for a store to
+    // release its chunk while the other already handles the next chunk.
     if (lane == 0) {
       const int g0 = warp >> 1;
       if (warp == 0) {
@@ -680,21 +681,19 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       }
       const uint64_t stream_once = l2_evict_first_policy();  // h is read here for the last time
       auto load_group = [&](int tile, int g) {
-        const int j = tile / tpp, rb = tile % tpp, c0 = g * 2, c1 = min(nchunk, c0 + 2);
-        mbar_expect_tx(h_full[g], (uint32_t)(c1 - c0) * 16384u);
-        for (int kc = c0; kc < c1; ++kc)
-          tma_load_3d_hint(smem_u32(htile + kc * 16384), &tmH, kc * 64, rb * 128, j, h_full[g], stream_once);
+        const int j = tile / tpp, rb = tile % tpp;
+        mbar_expect_tx(h_full[g], 16384u);
+        tma_load_3d_hint(smem_u32(htile + g * 16384), &tmH, g * 64, rb * 128, j, h_full[g], stream_once);
       };
       for (int g = g0; g < ngroups; g += 2) load_group(t_begin, g);
       uint32_t ph = 0;
       for (int tile = t_begin; tile < t_end && !failed; ++tile) {
         const int j = tile / tpp, rb = tile % tpp;
         for (int g = g0; g < ngroups; g += 2) {
-          // delta1 has replaced h in group g: store it, and once the store has read shared memory bring the
-          // next tile's h into the same chunks
+          // delta1 has replaced h in chunk g: store it, and once the store has read shared memory bring the
+          // next tile's h into the same chunk
           if (!mbar_wait(m_done[g], ph)) { failed = true; break; }
-          const int c0 = g * 2, c1 = min(nchunk, c0 + 2);
-          for (int kc = c0; kc < c1; ++kc) tma_store_3d(&tmD1, kc * 64, rb * 128, j, smem_u32(htile + kc * 16384));
+          tma_store_3d(&tmD1, g * 64, rb * 128, j, smem_u32(htile + g * 16384));
           tma_store_commit_and_wait_read();
           if (tile + 1 < t_end) load_group(tile + 1, g);
         }
@@ -711,7 +710,8 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
         for (int g = 0; g < ngroups && !failed; ++g) {
           if (!mbar_wait_warp(h_full[g], ph)) { failed = true; break; }
           tc_fence_after();
-          for (int kc = g * 2; kc < min(nchunk, g * 2 + 2); ++kc) {
+          {
+            const int kc = g;
             const uint64_t ad = smem_desc_sw128(smem_u32(htile + kc * 16384), 16, 1024);
             const uint64_t bd = smem_desc_sw128(smem_u32(w2t + kc * 2048), 16, 1024);
 #pragma unroll
@@ -825,14 +825,14 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       }
       uint32_t rr[64];  // this thread's 16 columns of each of the (up to) four chunks of a 256-column half
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
+      for (int g = 0; g < 8; ++g) {
         if (g >= ngroups || failed) break;
         // the threads read h themselves below: observe the completion of its TMA copies directly
         if (!mbar_wait(h_full[g], ph)) { failed = true; break; }
-        if ((g & 1) == 0) {  // first group of a half: fetch the half's accumulator and hand it back at once
+        if ((g & 3) == 0) {  // first chunk of a half: fetch the half's accumulator and hand it back at once
           if (!mbar_wait(d_full, dph)) { failed = true; break; }
           tc_fence_after();
-          const int hh = g >> 1, nlc = min(4, nchunk - hh * 4);
+          const int hh = g >> 2, nlc = min(4, nchunk - hh * 4);
 #pragma unroll
           for (int lc = 0; lc < 4; ++lc)
             if (lc < nlc) tmem_ld16_nowait(d_acc + lane_off + (uint32_t)(lc * 64 + part * 16), &rr[lc * 16]);
@@ -841,12 +841,13 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
           mbar_arrive(d_empty);
           dph ^= 1u;
         }
-        if (p.fuse && !mbar_wait(w_done[g], ph)) { failed = true; break; }  // the tensor cores are done with h
+        // the tensor cores are done with the 128 hidden units (two chunks) this chunk belongs to
+        if (p.fuse && (g & 1) == 0 && !mbar_wait(w_done[g >> 1], ph)) { failed = true; break; }
         const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int kc = g * 2 + cc;  // chunk of 64 hidden units
-          if (kc < nchunk) {
+        {
+          const int kc = g;  // chunk of 64 hidden units
+          {
             unsigned char *crow = htile + (size_t)kc * 16384 + row_off;
             uint4 hv[2];
 #pragma unroll
@@ -858,8 +859,8 @@ mlp_head_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
               uint32_t o[4];
 #pragma unroll
               for (int t2 = 0; t2 < 4; ++t2) {
-                // (g & 1) * 2 + cc = chunk inside the half; delta1 = (h > 0) ? value : 0 as a bf16 pair
-                const int e = (((g & 1) * 2 + cc) * 16) + i * 8 + t2 * 2;
+                // g & 3 = chunk inside the half; delta1 = (h > 0) ? value : 0 as a bf16 pair
+                const int e = ((g & 3) * 16) + i * 8 + t2 * 2;
                 const __nv_bfloat162 dv = __floats2bfloat162_rn(__uint_as_float(rr[e]), __uint_as_float(rr[e + 1]));
                 const __nv_bfloat162 hb = *reinterpret_cast<const __nv_bfloat162 *>(&hw4[t2]);
                 const __nv_bfloat162 dm = __hmul2(dv, __hgt2(hb, zero2));
@@ -1827,7 +1828,7 @@ cudaError_t launch_mlp_grad(int k, int rows, int d, int hidden, int C, const flo
   const int tpp = (rows + 127) / 128, hgrid = head_grid(k, rows, sms);
 
   const int nchunk = hidden / 64, nhalf = (hidden + 255) / 256;
-  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 512 + 1024;
+  const size_t head_tc_smem = (size_t)nchunk * 16384 + 16384 + (size_t)nhalf * 32768 + (size_t)nchunk * 2048 + 1024 + 1024;
   const bool head_tc = hidden % 64 == 0 && head_tc_smem <= 232448;
   const bool fuse_w2 = head_tc && hidden % 128 == 0;  // the head forms [dW2; db2] itself: no column of ones behind h
 
